@@ -1,0 +1,492 @@
+#!/usr/bin/env python
+"""Benchmark of the NVFP4 W4A4 linear-layer path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload mlp|quantize|gdn|linear]
+    python bench.py --impl reference ...        # times the CPU oracle instead
+
+Default workload ("mlp"): one step = one pass of the hot path over the MLP prefill
+pair of a 27B-class hybrid layer, M = 8192 tokens:
+    quantize X1 [8192 x 5120] -> fused gate/up GEMM (N = 2 x 17408, two segments,
+    separate global scales) -> quantize X2 [8192 x 17408] -> down GEMM (N = 5120).
+The headline value is GEMM FLOPs of the step divided by the WHOLE step time
+(quantization included).  The quantize kernel is also timed alone on the
+heavy-tailed 8192 x 5120 activation tensor and reported under "quantize".
+
+Prints one JSON line (rank 0).  Multi-GPU runs are independent replicas (the path
+has no exchange step): every rank runs the same step on its own GPU.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2609_04098_b200 import synth  # noqa: E402
+
+HIDDEN, INNER = synth.HIDDEN, synth.MLP_INNER
+NOMINAL_FP4_TFLOPS = 9000.0
+NOMINAL_HBM_GBS = 8000.0
+FP4_OVER_BF16 = 4.0          # nominal dense FP4 : bf16 tensor throughput on B200 (9 : 2.25 PFLOP/s)
+QUANT_BYTES_PER_ELEM = 2.0 + 0.5 + 1.0 / 16.0
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def ncu_traffic(name: str):
+    """DRAM bytes per launch from the committed ncu summary (profiles/traffic.json), or None."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    if not os.path.exists(path):
+        return None
+    with open(path) as f:
+        return json.load(f).get(name)
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.rows = []
+        self.proc = None
+        self.index = index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for r in self.rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------- workloads
+def gemm_flops(M, N, K):
+    return 2.0 * M * N * K
+
+
+class MlpPair:
+    """configs[2]: MLP prefill pair, M tokens."""
+    name = "mlp_prefill_pair"
+
+    def __init__(self, M=8192):
+        self.M = M
+        self.seg_gu = synth.make_segments((("gate", INNER, 0.02), ("up", INNER, 0.02)))
+        self.seg_d = synth.make_segments((("down", HIDDEN, 0.02),))
+        self.flops = gemm_flops(M, 2 * INNER, HIDDEN) + gemm_flops(M, HIDDEN, INNER)
+        self.quant_elems = M * HIDDEN + M * INNER
+        self.describe = ("configs[2] MLP prefill pair: M=%d, gate/up K=5120->N=2x17408 (2 segments), "
+                         "down K=17408->N=5120; activation quantize inside the step" % M)
+
+    def host_inputs(self, seed=0):
+        return {"x1": synth.prefill_activations(seed, 301, self.M, HIDDEN),
+                "x2": synth.prefill_activations(seed, 303, self.M, INNER),
+                "w_gu": synth.weights(seed, 302, self.seg_gu, HIDDEN),
+                "w_d": synth.weights(seed, 304, self.seg_d, INNER)}
+
+
+class GdnProj:
+    """configs[3]: fused GDN in-projection, six segments."""
+    name = "gdn_in_projection"
+
+    def __init__(self, M=8192):
+        self.M = M
+        self.segs = synth.make_segments(synth.GDN_SEGMENTS)
+        self.N = 16480
+        self.flops = gemm_flops(M, self.N, HIDDEN)
+        self.quant_elems = M * HIDDEN
+        self.describe = "configs[3] fused GDN in-projection: M=%d, K=5120, N=16480 in 6 segments" % M
+
+
+class OneLinear:
+    """configs[4]: one K=5120 -> N=6144 layer at a given M, quantize inside the timed call."""
+    name = "linear_5120_6144"
+
+    def __init__(self, M):
+        self.M = M
+        self.segs = synth.make_segments((("w", 6144, 0.02),))
+        self.N = 6144
+        self.flops = gemm_flops(M, self.N, HIDDEN)
+        self.quant_elems = M * HIDDEN
+        self.describe = "configs[4] linear K=5120->N=6144 at M=%d, quantize fused into the timed call" % M
+
+
+# --------------------------------------------------------------------------- GPU arm
+def run_gpu(args):
+    import torch
+    from paper_2609_04098_b200 import binding as nv
+    from paper_2609_04098_b200 import build as nvbuild
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    nvbuild.build()
+    nv.lib()
+    if args.variant:
+        nv.set_gemm_variant(args.variant)
+    peaks = measured_peaks()
+    fp4_peak = peaks["bf16_tflops_sustained"] * FP4_OVER_BF16
+    stream = torch.cuda.current_stream()
+
+    def up(bits):
+        return synth.to_torch_bf16(bits).to(dev)
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    result = {}
+    if args.workload == "mlp":
+        wl = MlpPair(args.tokens)
+        host = wl.host_inputs(args.seed)
+        x1, x2 = up(host["x1"]), up(host["x2"])
+        w_gu_c, w_gu_sf, g_gu = nv.nvfp4_quantize_weight(up(host["w_gu"]), wl.seg_gu)
+        w_d_c, w_d_sf, g_d = nv.nvfp4_quantize_weight(up(host["w_d"]), wl.seg_d)
+        g1, g2 = nv.nvfp4_calibrate(x1), nv.nvfp4_calibrate(x2)     # static activation scales (offline)
+        q1 = nv.alloc_quantized(wl.M, HIDDEN, dev)
+        q2 = nv.alloc_quantized(wl.M, INNER, dev)
+        y1 = torch.empty((wl.M, 2 * INNER), dtype=torch.bfloat16, device=dev)
+        y2 = torch.empty((wl.M, HIDDEN), dtype=torch.bfloat16, device=dev)
+        ws = nv.alloc_workspace(dev)
+        torch.cuda.synchronize()
+
+        def step(marks=None):
+            if marks is not None:
+                marks[0].record(stream)
+            nv.nvfp4_quantize_act(x1, g1, out=q1)
+            if marks is not None:
+                marks[1].record(stream)
+            nv.nvfp4_linear(q1[0], q1[1], g1, w_gu_c, w_gu_sf, wl.seg_gu, g_gu, ws, out=y1)
+            if marks is not None:
+                marks[2].record(stream)
+            nv.nvfp4_quantize_act(x2, g2, out=q2)
+            if marks is not None:
+                marks[3].record(stream)
+            nv.nvfp4_linear(q2[0], q2[1], g2, w_d_c, w_d_sf, wl.seg_d, g_d, ws, out=y2)
+            if marks is not None:
+                marks[4].record(stream)
+
+        gemm_slots, quant_slots, gemm_per_step = ((1, 2), (3, 4)), ((0, 1), (2, 3)), 2
+        h2d_tensors = [synth.to_torch_bf16(host["x1"]).pin_memory(), synth.to_torch_bf16(host["x2"]).pin_memory()]
+        d_inputs = [x1, x2]
+        d_result = y2
+        l2_note = "step touches >1 GB of distinct buffers (inputs larger than the 126 MB L2)"
+    elif args.workload in ("gdn", "linear"):
+        wl = GdnProj(args.tokens) if args.workload == "gdn" else OneLinear(args.tokens)
+        hx = synth.prefill_activations(args.seed, 401, wl.M, HIDDEN)
+        hw = synth.weights(args.seed, 402, wl.segs, HIDDEN)
+        # rotate through enough distinct activation/output sets to exceed L2
+        per_set = wl.M * HIDDEN * 2 + wl.M * wl.N * 2
+        nset = max(1, min(8, int(np.ceil(300e6 / per_set))))
+        xs = [up(hx) for _ in range(nset)]
+        w_c, w_sf, g_w = nv.nvfp4_quantize_weight(up(hw), wl.segs)
+        g1 = nv.nvfp4_calibrate(xs[0])
+        ys = [torch.empty((wl.M, wl.N), dtype=torch.bfloat16, device=dev) for _ in range(nset)]
+        wss = [nv.alloc_workspace(dev, wl.M, wl.N, HIDDEN, len(wl.segs), fused=True) for _ in range(nset)]
+        torch.cuda.synchronize()
+        counter = [0]
+
+        def step(marks=None):
+            i = counter[0] % nset
+            counter[0] += 1
+            if marks is not None:
+                marks[0].record(stream)
+            nv.nvfp4_linear_bf16(xs[i], g1, w_c, w_sf, wl.segs, g_w, wss[i], out=ys[i])
+            if marks is not None:
+                marks[1].record(stream)
+
+        gemm_slots, quant_slots, gemm_per_step = (), (), 1
+        h2d_tensors = [synth.to_torch_bf16(hx).pin_memory()]
+        d_inputs = [xs[0]]
+        d_result = ys[0]
+        l2_note = "rotating %d activation/output sets (%.0f MB) between iterations" % (nset, nset * per_set / 1e6)
+    else:
+        raise SystemExit("unknown workload")
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+
+    # ---- device-resident timing
+    for _ in range(max(3, args.warmup)):
+        step()
+    torch.cuda.synchronize()
+    nmark = 5 if args.workload == "mlp" else 2
+    marks = [[ev() for _ in range(nmark)] for _ in range(args.steps)]
+    sampler = ClockSampler(local_rank)
+    launches0 = nv.launch_count()
+    barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    t_start, t_end = ev(), ev()
+    t_start.record(stream)
+    for i in range(args.steps):
+        step(marks[i])
+    t_end.record(stream)
+    torch.cuda.synchronize()
+    barrier()
+    clocks = sampler.stop()
+    launches = nv.launch_count() - launches0
+    total_ms = t_start.elapsed_time(t_end)
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([total_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = wl.flops * world / (ms_per_step * 1e-3) / 1e12
+
+    # per-kernel durations from the marks (same timed region)
+    def span(slots):
+        return sum(m[a].elapsed_time(m[b]) for m in marks for (a, b) in slots)
+    if args.workload == "mlp":
+        gemm_ms = span(gemm_slots) / (args.steps * gemm_per_step)         # average per GEMM launch
+        quant_ms = span(quant_slots) / (args.steps * 2)
+        gemm_flops_per_launch = wl.flops / gemm_per_step
+        achieved = gemm_flops_per_launch / (gemm_ms * 1e-3) / 1e12
+        quant_in_step_gbs = wl.quant_elems / 2 * QUANT_BYTES_PER_ELEM / (quant_ms * 1e-3) / 1e9
+    else:
+        gemm_ms = ms_per_step
+        achieved = wl.flops / (gemm_ms * 1e-3) / 1e12
+        quant_in_step_gbs = None
+    roofline = {"kernel": "gemm_kernel (tcgen05 block-scaled FP4)", "bound": "tensor",
+                "achieved": round(achieved, 2), "peak": round(fp4_peak, 1), "unit": "TFLOP/s",
+                "frac": round(achieved / fp4_peak, 4),
+                "peak_basis": "%s bf16 sustained %.1f TFLOP/s x %.0f (nominal FP4:bf16 ratio)" % (
+                    peaks["source"], peaks["bf16_tflops_sustained"], FP4_OVER_BF16),
+                "frac_of_nominal_9pf": round(achieved / NOMINAL_FP4_TFLOPS, 4),
+                "avg_launch_ms": round(gemm_ms, 4),
+                "traffic": ncu_traffic("gemm_kernel")}
+    result["roofline"] = roofline
+
+    # ---- the quantize kernel alone on the heavy-tailed activation tensor (configs[1])
+    if rank == 0 and not args.skip_quantize:
+        hq = synth.config2_activations(args.seed)
+        nbuf = 6                                           # 6 x 84 MB inputs: larger than L2
+        xq = [up(hq) for _ in range(nbuf)]
+        gq = nv.nvfp4_calibrate(xq[0])
+        outs = [nv.alloc_quantized(8192, HIDDEN, dev) for _ in range(nbuf)]
+        for i in range(2 * nbuf):
+            nv.nvfp4_quantize_act(xq[i % nbuf], gq, out=outs[i % nbuf])
+        torch.cuda.synchronize()
+        reps = 10 * nbuf
+        e0, e1 = ev(), ev()
+        e0.record(stream)
+        for i in range(reps):
+            nv.nvfp4_quantize_act(xq[i % nbuf], gq, out=outs[i % nbuf])
+        e1.record(stream)
+        torch.cuda.synchronize()
+        q_ms = e0.elapsed_time(e1) / reps
+        q_bytes = 8192 * HIDDEN * QUANT_BYTES_PER_ELEM
+        q_gbs = q_bytes / (q_ms * 1e-3) / 1e9
+        c0, c1 = ev(), ev()
+        c0.record(stream)
+        for i in range(reps):
+            nv.nvfp4_calibrate(xq[i % nbuf], g=gq)
+        c1.record(stream)
+        torch.cuda.synchronize()
+        cal_ms = c0.elapsed_time(c1) / reps
+        result["quantize"] = {
+            "workload": "configs[1] activation quantize 8192x5120 bf16, heavy-tailed; %d rotating buffers" % nbuf,
+            "metric": "act_quantize_gbs", "value": round(q_gbs, 1), "unit": "GB/s", "us_per_call": round(q_ms * 1e3, 2),
+            "roofline": {"kernel": "quantize_kernel", "bound": "hbm", "achieved": round(q_gbs, 1),
+                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(q_gbs / peaks["hbm_gbs"], 4),
+                         "peak_basis": "%s copy bandwidth" % peaks["source"],
+                         "frac_of_nominal_8tbs": round(q_gbs / NOMINAL_HBM_GBS, 4),
+                         "traffic": ncu_traffic("quantize_kernel")},
+            "calibrate_gbs": round(8192 * HIDDEN * 2 / (cal_ms * 1e-3) / 1e9, 1),
+            "in_step_gbs": None if quant_in_step_gbs is None else round(quant_in_step_gbs, 1)}
+        del xq, outs
+
+    # ---- end to end: host buffers in, result back, through the same calls
+    e2e_steps = max(1, min(args.steps, 5))
+    h_out = torch.empty_like(d_result, device="cpu").pin_memory()
+    h2d_bytes = sum(t.numel() * t.element_size() for t in h2d_tensors)
+    d2h_bytes = h_out.numel() * h_out.element_size()
+
+    def e2e_step():
+        for src, dst in zip(h2d_tensors, d_inputs):
+            dst.copy_(src, non_blocking=True)
+        step()
+        h_out.copy_(d_result, non_blocking=True)
+
+    e2e_step()
+    torch.cuda.synchronize()
+    barrier()
+    s0, s1 = ev(), ev()
+    s0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    s1.record(stream)
+    torch.cuda.synchronize()
+    e2e_ms = s0.elapsed_time(s1) / e2e_steps
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([e2e_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    result["e2e"] = {"value": round(wl.flops * world / (e2e_ms * 1e-3) / 1e12, 2), "unit": "TFLOP/s",
+                     "ms_per_step": round(e2e_ms, 3), "h2d_bytes_per_step": h2d_bytes,
+                     "d2h_bytes_per_step": d2h_bytes}
+    status = nv.device_status(ws if args.workload == "mlp" else wss[0])
+    if status != 0:
+        raise SystemExit("device status %d after the timed region" % status)
+
+    if rank == 0:
+        if not args.skip_cpu:
+            result["cpu_baseline"] = cpu_baseline(wl, target_s=args.cpu_seconds, seed=args.seed)
+        line = {"metric": "nvfp4_w4a4_linear_tflops", "value": round(value, 2), "unit": "TFLOP/s",
+                "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
+                "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "nvfp4 (e2m1 x e4m3 block scales, f32 accumulate, bf16 out)",
+                "data": "synthetic (seeded; shapes and statistics of the paper's 27B hybrid model)",
+                "config": {"workload": wl.describe, "tokens": wl.M, "l2": l2_note,
+                           "parallelism": "replicas only" if world > 1 else "single GPU",
+                           "gemm_variant": args.variant or "auto"},
+                "gpu_launches": int(launches), "clocks": clocks}
+        line.update(result)
+        print(json.dumps(line))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+# --------------------------------------------------------------------------- CPU oracle arm
+def cpu_baseline(wl, target_s=15.0, seed=0):
+    """The oracle as it stands, timed on a bounded sample of the same workload:
+    quantize R activation rows, then the exact GEMM of those rows against a slice of
+    the first layer's weight rows."""
+    import oracle
+    K = HIDDEN
+    segs = wl.seg_gu if hasattr(wl, "seg_gu") else wl.segs
+    n_full = sum(s.count for s in segs)
+    ncols = min(n_full, 2048)
+    w = synth.weights(seed, 302, synth.make_segments((("w", ncols, 0.02),)), K)
+    _, gw = oracle.calibrate(w)
+    wc, wsf = oracle.quantize(w, oracle.row_scales(ncols, g=gw))
+    gcol = np.full(ncols, gw, np.float32)
+
+    def run(rows):
+        x = synth.prefill_activations(seed, 301, rows, K)
+        t0 = time.perf_counter()
+        _, ga = oracle.calibrate(x)
+        ac, asf = oracle.quantize(x, oracle.row_scales(rows, g=ga))
+        oracle.gemm(ac, asf, ga, wc, wsf, gcol)
+        return time.perf_counter() - t0
+
+    t_small = run(8)
+    rows = int(max(8, min(1024, 8 * target_s / max(t_small, 1e-3))))
+    t = run(rows)
+    flops = gemm_flops(rows, ncols, K)
+    return {"value": round(flops / t / 1e12, 6), "unit": "TFLOP/s", "cores": oracle.num_threads(),
+            "kind": "oracle", "seconds": round(t, 2),
+            "sample": "quantize + exact GEMM of %d token rows x %d weight rows (K=%d) of the first layer" % (
+                rows, ncols, K)}
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle on the same metric and workload, each step a
+    bounded sample.  Rank 0 only."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    wl = {"mlp": MlpPair, "gdn": GdnProj, "linear": OneLinear}[args.workload](args.tokens)
+    per_step_s = max(2.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    for _ in range(args.warmup):
+        cpu_baseline(wl, target_s=per_step_s / 4, seed=args.seed)
+    vals, secs, last = [], [], None
+    for _ in range(args.steps):
+        last = cpu_baseline(wl, target_s=per_step_s, seed=args.seed)
+        vals.append(last["value"])
+        secs.append(last["seconds"])
+    value = float(np.mean(vals))
+    line = {"impl": "reference", "metric": "nvfp4_w4a4_linear_tflops", "value": round(value, 6), "unit": "TFLOP/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": round(1e3 * float(np.mean(secs)), 1), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "int64/f64 (exact)", "data": "synthetic (seeded)",
+            "config": {"workload": wl.describe, "tokens": wl.M},
+            "cpu_baseline": {"value": round(value, 6), "unit": "TFLOP/s", "kind": "oracle",
+                             "cores": last["cores"], "sample": last["sample"]},
+            "e2e": {"value": round(value, 6), "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="mlp", choices=["mlp", "gdn", "linear"])
+    ap.add_argument("--tokens", type=int, default=8192)
+    ap.add_argument("--variant", type=int, default=0, help="GEMM tile variant (0 = auto)")
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--skip-cpu", action="store_true")
+    ap.add_argument("--skip-quantize", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,192 @@
+/*
+ * nvfp4.h -- C ABI of the B200 (sm_100a) NVFP4 W4A4 linear-layer library.
+ *
+ * The path (paper: Background, "NVFP4"; Section 6, "Per-module calibration vs.
+ * fused-GEMM scaling"):
+ *
+ *   bf16 activations --nvfp4_quantize_act--> E2M1 codes + one E4M3 scale per
+ *   16-element block (+ an FP32 per-tensor global scale)
+ *   --nvfp4_linear--> block-scaled FP4 GEMM against weights quantized once by
+ *   nvfp4_quantize_weight, with ONE GLOBAL SCALE PER FUSED MODULE applied to that
+ *   module's slice of output columns in the epilogue.
+ *
+ * Conventions for every entry point
+ *   - Pointers named d_* are DEVICE pointers; everything else is host memory.
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = the
+ *     legacy default stream).  No call synchronises the device except
+ *     nvfp4_device_status.  No call allocates or frees device memory.
+ *   - The caller owns every buffer; the library keeps no pointer after the call
+ *     returns other than cached TMA descriptors keyed by (address, shape), which
+ *     hold no reference.
+ *   - Host-detectable misuse returns a status before anything is launched.
+ *     Nothing throws across this boundary.
+ *   - Quantized tensor layout:  codes are row-major [rows, K/2] bytes, element k
+ *     of a row in byte k/2, low nibble for even k.  Scale bytes (E4M3, one per
+ *     16 consecutive k) are stored either
+ *       NVFP4_SF_LINEAR: row-major [rows, K/16], or
+ *       NVFP4_SF_MMA:    the order the block-scaled tensor-core instruction reads:
+ *                        512-byte atoms of 128 rows x 4 blocks, byte offset of
+ *                        (r, b) inside its atom = (r%32)*16 + ((r%128)/32)*4 + b%4,
+ *                        atoms of one 128-row band contiguous along K; rows are
+ *                        padded to a multiple of 128 and blocks to a multiple of
+ *                        4, padding bytes are 0x00.
+ *     nvfp4_sf_bytes gives the buffer size for either.
+ *   - Global scales are "decode direction": x ~= e2m1 * e4m3 * g.  They must be
+ *     finite and > 0.
+ */
+#ifndef NVFP4_H_
+#define NVFP4_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    NVFP4_OK = 0,
+    NVFP4_ERR_NULL = 1,        /* a required pointer is NULL */
+    NVFP4_ERR_SHAPE = 2,       /* a size is negative, or K is not a multiple of 16 (GEMM: 64) */
+    NVFP4_ERR_ALIGN = 3,       /* a pointer or leading dimension breaks the stated alignment */
+    NVFP4_ERR_SEGMENTS = 4,    /* segment table is not a sorted, gap-free cover of [0, N) */
+    NVFP4_ERR_WORKSPACE = 5,   /* workspace missing or too small */
+    NVFP4_ERR_ARCH = 6,        /* current device is not compute capability 10.x */
+    NVFP4_ERR_CUDA = 7,        /* a CUDA runtime/driver call or a launch failed */
+    NVFP4_ERR_TIMEOUT = 8,     /* a bounded wait inside a kernel ran out (see nvfp4_device_status) */
+    NVFP4_ERR_LAYOUT = 9       /* unknown scale layout / the GEMM needs NVFP4_SF_MMA */
+} nvfp4_status;
+
+/* One fused module's slice of the output columns (= rows of the weight matrix). */
+typedef struct {
+    int64_t col_begin;
+    int64_t col_count;
+} nvfp4_segment;
+
+#define NVFP4_MAX_SEGMENTS 32
+
+typedef enum { NVFP4_SF_LINEAR = 0, NVFP4_SF_MMA = 1 } nvfp4_sf_layout;
+
+/* flags for nvfp4_linear* */
+#define NVFP4_OUT_BF16 0u     /* Y is bf16 (default)                                  */
+#define NVFP4_OUT_F32  1u     /* Y is float32 (testing aid: no output rounding)       */
+
+/* Size in bytes of the scale buffer for a [rows, K] tensor in `layout` (K % 16 == 0). */
+size_t nvfp4_sf_bytes(int64_t rows, int64_t K, nvfp4_sf_layout layout);
+
+/*
+ * Global-scale calibration (paper: one FP32 scale per tensor / per linear module;
+ * the value amax/(6*448) makes the block that holds the tensor maximum use the
+ * largest E4M3 scale).
+ *   d_x     bf16 [rows, cols], row stride ld elements (ld >= cols)
+ *   d_g     out: *d_g = amax / 2688 in binary32, or 1.0f if the tensor is all zero
+ *   d_amax  out, optional (may be NULL): max |x|
+ * Errors: NULL d_x/d_g, negative sizes, ld < cols.  rows*cols == 0 gives g = 1.
+ */
+nvfp4_status nvfp4_calibrate(const void* d_x, int64_t rows, int64_t cols, int64_t ld,
+                             float* d_g, float* d_amax, void* stream);
+
+/*
+ * On-the-fly activation quantization (paper: Background, "NVFP4": E2M1 values, one
+ * E4M3 scale per 16-element block set to blockmax/6, one FP32 scale per tensor).
+ * Per block of 16 consecutive k, in binary32 with round-to-nearest-even and no
+ * fused multiply-add:
+ *     s8   = e4m3_rne_sat( bmax * (1 / (6 * g)) )
+ *     code = e2m1_rne_sat( x * (1 / (e4m3(s8) * g)) )     (all codes 0 if s8 == 0)
+ *   d_x      bf16 [M, K], row stride ld elements; 16-byte aligned, ld % 8 == 0
+ *   d_g      in: the tensor's global scale (device scalar)
+ *   d_codes  out: [M, K/2] bytes, 16-byte aligned
+ *   d_sf     out: nvfp4_sf_bytes(M, K, layout) bytes (padding is written as zero)
+ * Errors: NULL pointers, K % 16 != 0, misalignment, unknown layout.  M == 0 is a no-op.
+ */
+nvfp4_status nvfp4_quantize_act(const void* d_x, int64_t M, int64_t K, int64_t ld,
+                                const float* d_g, uint8_t* d_codes, uint8_t* d_sf,
+                                nvfp4_sf_layout layout, void* stream);
+
+/*
+ * Offline weight quantization, same format, blocks along K, with one global scale
+ * per fused module (paper: Section 6 -- the calibration tool keeps one FP32 global
+ * scale per linear module; the modules are later served as one fused GEMM).
+ *   d_w      bf16 [N, K], row stride ld; rows are the output features
+ *   segs     host array of nseg segments covering rows [0, N) in order, no gaps
+ *   d_g_seg  device float[nseg]: INPUT when calibrate_segments == 0; OUTPUT
+ *            (per-segment amax/2688) when calibrate_segments != 0
+ * Errors: as nvfp4_quantize_act, plus NVFP4_ERR_SEGMENTS, nseg < 1 or > NVFP4_MAX_SEGMENTS.
+ */
+nvfp4_status nvfp4_quantize_weight(const void* d_w, int64_t N, int64_t K, int64_t ld,
+                                   const nvfp4_segment* segs, int nseg, float* d_g_seg,
+                                   int calibrate_segments, uint8_t* d_codes, uint8_t* d_sf,
+                                   nvfp4_sf_layout layout, void* stream);
+
+/*
+ * The W4A4 linear layer (paper: Background, "NVFP4": the GEMM runs on 4-bit tensor
+ * cores; Section 6: per-module global scales meeting in one fused GEMM -- here each
+ * segment of output columns gets its own global scale in the epilogue, which is
+ * exact, instead of one scale for the whole fused GEMM):
+ *     Y[m, n] = round_out( (sum_k a_hat[m,k] * w_hat[n,k]) * g_a * g_seg[seg(n)] )
+ * where a_hat/w_hat are code*block-scale products, accumulated in FP32 on the tensor
+ * cores.
+ *   d_a_codes/d_a_sf   activations [M, K] as written by nvfp4_quantize_act with NVFP4_SF_MMA
+ *   d_w_codes/d_w_sf   weights [N, K] as written by nvfp4_quantize_weight with NVFP4_SF_MMA
+ *   d_g_a              device scalar; d_g_seg device float[nseg]
+ *   segs               host array (copied into the launch; need not outlive the call)
+ *   d_y                out [M, N], row stride ldy elements, bf16 or float per `flags`
+ *   d_workspace        nvfp4_linear_workspace_bytes(...) bytes, 16-byte aligned; its first
+ *                      word is a status flag read by nvfp4_device_status
+ * Requirements: K % 64 == 0; code pointers 16-byte aligned; scale pointers 16-byte aligned.
+ * Errors: see nvfp4_status; M == 0 or N == 0 is a no-op.
+ */
+nvfp4_status nvfp4_linear(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const float* d_g_a,
+                          int64_t M, int64_t K,
+                          const uint8_t* d_w_codes, const uint8_t* d_w_sf, int64_t N,
+                          const nvfp4_segment* segs, const float* d_g_seg, int nseg,
+                          void* d_y, int64_t ldy, uint32_t flags,
+                          void* d_workspace, size_t workspace_bytes, void* stream);
+
+size_t nvfp4_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int nseg);
+
+/*
+ * The same layer fed with bf16 activations: quantization runs inside the call
+ * (paper: Section 9, "Decode overhead" -- activation quantization is the overhead
+ * that matters at small batch), codes and scales live in the workspace.
+ *   d_x   bf16 [M, K], row stride ldx, 16-byte aligned, ldx % 8 == 0
+ */
+nvfp4_status nvfp4_linear_bf16(const void* d_x, int64_t ldx, const float* d_g_a,
+                               int64_t M, int64_t K,
+                               const uint8_t* d_w_codes, const uint8_t* d_w_sf, int64_t N,
+                               const nvfp4_segment* segs, const float* d_g_seg, int nseg,
+                               void* d_y, int64_t ldy, uint32_t flags,
+                               void* d_workspace, size_t workspace_bytes, void* stream);
+
+size_t nvfp4_linear_bf16_workspace_bytes(int64_t M, int64_t N, int64_t K, int nseg);
+
+/*
+ * Clears the status word of a workspace (enqueue before the first nvfp4_linear* that
+ * uses it; the kernels only ever set it).
+ */
+nvfp4_status nvfp4_workspace_reset(void* d_workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Synchronises `stream` and returns the status word of the workspace: NVFP4_OK, or
+ * NVFP4_ERR_TIMEOUT if a kernel gave up on one of its bounded waits (its output is
+ * then unspecified; the CUDA context stays usable).
+ */
+nvfp4_status nvfp4_device_status(const void* d_workspace, void* stream);
+
+/* Number of this library's kernel launches enqueued so far by this process. */
+uint64_t nvfp4_launch_count(void);
+
+/*
+ * Tile shape of the GEMM kernel: 0 = choose from the problem size (default),
+ * otherwise one of the values nvfp4_status_string(NVFP4_OK)'s sibling
+ * nvfp4_gemm_variants() lists.  Process-wide; meant for benchmarking.
+ */
+nvfp4_status nvfp4_set_gemm_variant(int variant);
+const char* nvfp4_gemm_variants(void);
+
+const char* nvfp4_status_string(nvfp4_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NVFP4_H_ */

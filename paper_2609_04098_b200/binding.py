@@ -1,0 +1,219 @@
+"""Python binding of the C ABI in ``include/nvfp4.h``: argument marshalling only.
+
+Every function takes torch CUDA tensors (device memory and streams are all that
+torch provides here), passes raw pointers and sizes to the library and raises
+``Nvfp4Error`` on a non-zero status.  There is no CPU or torch fallback: if the
+library has not been built the first call fails.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libnvfp4_b200.so")
+
+SF_LINEAR = 0
+SF_MMA = 1
+OUT_BF16 = 0
+OUT_F32 = 1
+MAX_SEGMENTS = 32
+
+EXPORTS = (
+    "nvfp4_sf_bytes", "nvfp4_calibrate", "nvfp4_quantize_act", "nvfp4_quantize_weight",
+    "nvfp4_linear", "nvfp4_linear_workspace_bytes", "nvfp4_linear_bf16",
+    "nvfp4_linear_bf16_workspace_bytes", "nvfp4_workspace_reset", "nvfp4_device_status",
+    "nvfp4_launch_count", "nvfp4_set_gemm_variant", "nvfp4_gemm_variants", "nvfp4_status_string",
+)
+
+
+class Nvfp4Error(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s: status %d (%s)" % (where, status, status_string(status)))
+
+
+class _Segment(ctypes.Structure):
+    _fields_ = [("col_begin", ctypes.c_int64), ("col_count", ctypes.c_int64)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load the CUDA library (built by ``paper_2609_04098_b200.build``); no fallback."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError("CUDA library missing: %s -- run `python -m paper_2609_04098_b200.build`" % LIB_PATH)
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i64, i32, u32, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_uint32, ctypes.c_size_t
+    segp = ctypes.POINTER(_Segment)
+    L.nvfp4_sf_bytes.restype = sz
+    L.nvfp4_sf_bytes.argtypes = [i64, i64, i32]
+    L.nvfp4_calibrate.restype = i32
+    L.nvfp4_calibrate.argtypes = [vp, i64, i64, i64, vp, vp, vp]
+    L.nvfp4_quantize_act.restype = i32
+    L.nvfp4_quantize_act.argtypes = [vp, i64, i64, i64, vp, vp, vp, i32, vp]
+    L.nvfp4_quantize_weight.restype = i32
+    L.nvfp4_quantize_weight.argtypes = [vp, i64, i64, i64, segp, i32, vp, i32, vp, vp, i32, vp]
+    L.nvfp4_linear.restype = i32
+    L.nvfp4_linear.argtypes = [vp, vp, vp, i64, i64, vp, vp, i64, segp, vp, i32, vp, i64, u32, vp, sz, vp]
+    L.nvfp4_linear_workspace_bytes.restype = sz
+    L.nvfp4_linear_workspace_bytes.argtypes = [i64, i64, i64, i32]
+    L.nvfp4_linear_bf16.restype = i32
+    L.nvfp4_linear_bf16.argtypes = [vp, i64, vp, i64, i64, vp, vp, i64, segp, vp, i32, vp, i64, u32, vp, sz, vp]
+    L.nvfp4_linear_bf16_workspace_bytes.restype = sz
+    L.nvfp4_linear_bf16_workspace_bytes.argtypes = [i64, i64, i64, i32]
+    L.nvfp4_workspace_reset.restype = i32
+    L.nvfp4_workspace_reset.argtypes = [vp, sz, vp]
+    L.nvfp4_device_status.restype = i32
+    L.nvfp4_device_status.argtypes = [vp, vp]
+    L.nvfp4_launch_count.restype = ctypes.c_uint64
+    L.nvfp4_launch_count.argtypes = []
+    L.nvfp4_set_gemm_variant.restype = i32
+    L.nvfp4_set_gemm_variant.argtypes = [i32]
+    L.nvfp4_gemm_variants.restype = ctypes.c_char_p
+    L.nvfp4_gemm_variants.argtypes = []
+    L.nvfp4_status_string.restype = ctypes.c_char_p
+    L.nvfp4_status_string.argtypes = [i32]
+    _lib = L
+    return L
+
+
+def status_string(status: int) -> str:
+    return lib().nvfp4_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != 0:
+        raise Nvfp4Error(status, where)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _segments(segments: Sequence[Tuple[int, int]]):
+    arr = (_Segment * max(1, len(segments)))()
+    for i, (b, c) in enumerate(segments):
+        arr[i].col_begin, arr[i].col_count = int(b), int(c)
+    return arr
+
+
+def seg_pairs(segments) -> Sequence[Tuple[int, int]]:
+    """Accept (begin, count) pairs or objects with .begin/.count."""
+    return [(s.begin, s.count) if hasattr(s, "begin") else (int(s[0]), int(s[1])) for s in segments]
+
+
+def launch_count() -> int:
+    return int(lib().nvfp4_launch_count())
+
+
+def set_gemm_variant(variant: int) -> None:
+    _check(lib().nvfp4_set_gemm_variant(int(variant)), "nvfp4_set_gemm_variant")
+
+
+def sf_bytes(rows: int, K: int, layout: int = SF_MMA) -> int:
+    return int(lib().nvfp4_sf_bytes(rows, K, layout))
+
+
+def nvfp4_calibrate(x: torch.Tensor, g: Optional[torch.Tensor] = None, amax: Optional[torch.Tensor] = None,
+                    stream=None) -> torch.Tensor:
+    """amax -> global scale g = amax/(6*448) (device scalar, float32)."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
+    if g is None:
+        g = torch.empty(1, dtype=torch.float32, device=x.device)
+    _check(lib().nvfp4_calibrate(_ptr(x), x.shape[0], x.shape[1], x.stride(0), _ptr(g), _ptr(amax),
+                                 _stream(stream)), "nvfp4_calibrate")
+    return g
+
+
+def alloc_quantized(rows: int, K: int, device, layout: int = SF_MMA):
+    codes = torch.empty((rows, K // 2), dtype=torch.uint8, device=device)
+    sf = torch.empty(max(1, sf_bytes(rows, K, layout)), dtype=torch.uint8, device=device)
+    return codes, sf
+
+
+def nvfp4_quantize_act(x: torch.Tensor, g: torch.Tensor, layout: int = SF_MMA, out=None, stream=None):
+    """bf16 [M, K] -> (codes u8 [M, K/2], scale bytes u8 [nvfp4_sf_bytes])."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
+    M, K = x.shape
+    codes, sf = out if out is not None else alloc_quantized(M, K, x.device, layout)
+    _check(lib().nvfp4_quantize_act(_ptr(x), M, K, x.stride(0), _ptr(g), _ptr(codes), _ptr(sf), layout,
+                                    _stream(stream)), "nvfp4_quantize_act")
+    return codes, sf
+
+
+def nvfp4_quantize_weight(w: torch.Tensor, segments, g_seg: Optional[torch.Tensor] = None,
+                          layout: int = SF_MMA, out=None, stream=None):
+    """bf16 [N, K] -> (codes, scale bytes, g_seg).  ``g_seg=None`` calibrates each
+    segment (amax/2688) on the device; otherwise the given per-segment scales are used."""
+    assert w.is_cuda and w.dtype == torch.bfloat16 and w.dim() == 2 and w.stride(1) == 1
+    N, K = w.shape
+    pairs = seg_pairs(segments)
+    calibrate = 0
+    if g_seg is None:
+        g_seg = torch.empty(len(pairs), dtype=torch.float32, device=w.device)
+        calibrate = 1
+    codes, sf = out if out is not None else alloc_quantized(N, K, w.device, layout)
+    _check(lib().nvfp4_quantize_weight(_ptr(w), N, K, w.stride(0), _segments(pairs), len(pairs), _ptr(g_seg),
+                                       calibrate, _ptr(codes), _ptr(sf), layout, _stream(stream)),
+           "nvfp4_quantize_weight")
+    return codes, sf, g_seg
+
+
+def alloc_workspace(device, M: int = 0, N: int = 0, K: int = 0, nseg: int = 1, fused: bool = False) -> torch.Tensor:
+    n = (lib().nvfp4_linear_bf16_workspace_bytes(M, N, K, nseg) if fused
+         else lib().nvfp4_linear_workspace_bytes(M, N, K, nseg))
+    ws = torch.zeros(int(n), dtype=torch.uint8, device=device)
+    return ws
+
+
+def nvfp4_linear(a_codes, a_sf, g_a, w_codes, w_sf, segments, g_seg, workspace, out=None,
+                 out_f32: bool = False, stream=None) -> torch.Tensor:
+    """Y[M, N] = (A_q . W_q^T) * g_a * g_seg[segment of n]; bf16 (or float32) output."""
+    M, K = a_codes.shape[0], a_codes.shape[1] * 2
+    N = w_codes.shape[0]
+    pairs = seg_pairs(segments)
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.float32 if out_f32 else torch.bfloat16, device=a_codes.device)
+    flags = OUT_F32 if out.dtype == torch.float32 else OUT_BF16
+    _check(lib().nvfp4_linear(_ptr(a_codes), _ptr(a_sf), _ptr(g_a), M, K, _ptr(w_codes), _ptr(w_sf), N,
+                              _segments(pairs), _ptr(g_seg), len(pairs), _ptr(out), out.stride(0), flags,
+                              _ptr(workspace), workspace.numel(), _stream(stream)), "nvfp4_linear")
+    return out
+
+
+def nvfp4_linear_bf16(x, g_a, w_codes, w_sf, segments, g_seg, workspace, out=None, out_f32: bool = False,
+                      stream=None) -> torch.Tensor:
+    """Same layer fed with bf16 activations; quantization happens inside the call."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
+    M, K = x.shape
+    N = w_codes.shape[0]
+    pairs = seg_pairs(segments)
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.float32 if out_f32 else torch.bfloat16, device=x.device)
+    flags = OUT_F32 if out.dtype == torch.float32 else OUT_BF16
+    _check(lib().nvfp4_linear_bf16(_ptr(x), x.stride(0), _ptr(g_a), M, K, _ptr(w_codes), _ptr(w_sf), N,
+                                   _segments(pairs), _ptr(g_seg), len(pairs), _ptr(out), out.stride(0), flags,
+                                   _ptr(workspace), workspace.numel(), _stream(stream)), "nvfp4_linear_bf16")
+    return out
+
+
+def workspace_reset(workspace: torch.Tensor, stream=None) -> None:
+    _check(lib().nvfp4_workspace_reset(_ptr(workspace), workspace.numel(), _stream(stream)), "nvfp4_workspace_reset")
+
+
+def device_status(workspace: torch.Tensor, stream=None) -> int:
+    """Synchronises the stream; 0 = ok, 8 = a bounded in-kernel wait ran out."""
+    return int(lib().nvfp4_device_status(_ptr(workspace), _stream(stream)))

@@ -1,0 +1,416 @@
+// Host side of the C ABI declared in include/nvfp4.h: argument checks, TMA
+// descriptor set-up (cached), tile-shape choice and launches.  No allocation,
+// no synchronisation (except nvfp4_device_status), nothing thrown.
+#include <atomic>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+#include <unordered_map>
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include "../../include/nvfp4.h"
+#include "gemm.cuh"
+#include "quantize.cuh"
+
+namespace nvfp4 {
+namespace {
+
+std::atomic<uint64_t> g_launches{0};
+std::atomic<int> g_variant{0};
+constexpr uint64_t kWaitLimitNs = 2000000000ull;   // every in-kernel wait gives up after 2 s
+
+inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+struct DeviceInfo {
+    int sm_count = 0;
+    int cc_major = 0;
+    bool ok = false;
+};
+
+DeviceInfo device_info() {
+    static std::mutex mu;
+    static std::unordered_map<int, DeviceInfo> cache;
+    int dev = 0;
+    DeviceInfo info;
+    if (cudaGetDevice(&dev) != cudaSuccess) return info;
+    std::lock_guard<std::mutex> lock(mu);
+    auto it = cache.find(dev);
+    if (it != cache.end()) return it->second;
+    if (cudaDeviceGetAttribute(&info.sm_count, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&info.cc_major, cudaDevAttrComputeCapabilityMajor, dev) == cudaSuccess)
+        info.ok = true;
+    cache[dev] = info;
+    return info;
+}
+
+nvfp4_status check_arch(DeviceInfo& info) {
+    info = device_info();
+    if (!info.ok) return NVFP4_ERR_CUDA;
+    if (info.cc_major != 10) return NVFP4_ERR_ARCH;
+    return NVFP4_OK;
+}
+
+nvfp4_status check_segments(const nvfp4_segment* segs, int nseg, int64_t N) {
+    if (segs == nullptr) return NVFP4_ERR_NULL;
+    if (nseg < 1 || nseg > NVFP4_MAX_SEGMENTS) return NVFP4_ERR_SEGMENTS;
+    int64_t pos = 0;
+    for (int i = 0; i < nseg; ++i) {
+        if (segs[i].col_begin != pos || segs[i].col_count <= 0) return NVFP4_ERR_SEGMENTS;
+        pos += segs[i].col_count;
+    }
+    return pos == N ? NVFP4_OK : NVFP4_ERR_SEGMENTS;
+}
+
+// ---------------------------------------------------------------- tensor maps
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = []() -> EncodeTiledFn {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            return nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+struct MapKey {
+    const void* ptr;
+    int64_t rows, kbytes;
+    int box_rows, dev;
+    bool operator==(const MapKey& o) const {
+        return ptr == o.ptr && rows == o.rows && kbytes == o.kbytes && box_rows == o.box_rows && dev == o.dev;
+    }
+};
+struct MapKeyHash {
+    size_t operator()(const MapKey& k) const {
+        size_t h = std::hash<const void*>()(k.ptr);
+        h ^= std::hash<int64_t>()(k.rows * 1315423911ll + k.kbytes) + 0x9e3779b97f4a7c15ull + (h << 6) + (h >> 2);
+        return h ^ static_cast<size_t>(k.box_rows * 31 + k.dev);
+    }
+};
+
+// codes [rows, K/2] bytes, tiles of box_rows x 128 bytes, 128-byte swizzle, zero fill outside
+nvfp4_status codes_tensor_map(const uint8_t* d_codes, int64_t rows, int64_t K, int box_rows, CUtensorMap* out) {
+    static std::mutex mu;
+    static std::unordered_map<MapKey, CUtensorMap, MapKeyHash> cache;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    MapKey key{d_codes, rows, K / 2, box_rows, dev};
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        auto it = cache.find(key);
+        if (it != cache.end()) { *out = it->second; return NVFP4_OK; }
+    }
+    EncodeTiledFn enc = encode_fn();
+    if (enc == nullptr) return NVFP4_ERR_CUDA;
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(K / 2), static_cast<cuuint64_t>(rows)};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(K / 2)};
+    const cuuint32_t box[2] = {static_cast<cuuint32_t>(kBKBytes), static_cast<cuuint32_t>(box_rows)};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(d_codes), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return NVFP4_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (cache.size() > 4096) cache.clear();
+    cache[key] = *out;
+    return NVFP4_OK;
+}
+
+// ---------------------------------------------------------------- GEMM launch
+template <int BN, int ACC, int STAGES>
+nvfp4_status launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, GemmParams& p, int sm_count,
+                         cudaStream_t stream) {
+    using C = GemmCfg<BN, ACC, STAGES>;
+    static std::mutex mu;
+    static std::unordered_map<int, bool> configured;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        if (!configured[dev]) {
+            if (cudaFuncSetAttribute(gemm_kernel<BN, ACC, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     C::SMEM_BYTES) != cudaSuccess)
+                return NVFP4_ERR_CUDA;
+            configured[dev] = true;
+        }
+    }
+    p.n_tiles = (p.N + BN - 1) / BN;
+    const int64_t tiles = static_cast<int64_t>(p.m_tiles) * p.n_tiles;
+    const int grid = static_cast<int>(tiles < sm_count ? tiles : sm_count);
+    gemm_kernel<BN, ACC, STAGES><<<grid, kGemmThreads, C::SMEM_BYTES, stream>>>(tmA, tmB, p);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+}
+
+int choose_variant(int64_t M, int64_t N) {
+    const int forced = g_variant.load(std::memory_order_relaxed);
+    if (forced != 0) return forced;
+    (void)M;
+    return N >= 256 ? 256 : 128;
+}
+
+nvfp4_status quantize_impl(const void* d_x, int64_t M, int64_t K, int64_t ld, const float* d_g,
+                           const SegTable& segs, uint8_t* d_codes, uint8_t* d_sf, nvfp4_sf_layout layout,
+                           const DeviceInfo& info, cudaStream_t stream) {
+    const int64_t chunks = (K + 255) / 256;
+    if (M * chunks >= (1ll << 31) || K >= (1ll << 31)) return NVFP4_ERR_SHAPE;
+    if (layout == NVFP4_SF_MMA && (M % 128) != 0) {
+        // rows of the last 128-row band that the tensor does not have must read as zero scales
+        const int64_t katoms = (K / 16 + 3) / 4;
+        if (cudaMemsetAsync(d_sf + (M / 128) * katoms * 512, 0, static_cast<size_t>(katoms * 512), stream) !=
+            cudaSuccess)
+            return NVFP4_ERR_CUDA;
+    }
+    const int32_t total = static_cast<int32_t>(M * chunks);
+    constexpr int kUnroll = 4;
+    const int64_t warps_needed = (total + kUnroll - 1) / kUnroll;
+    int64_t blocks = (warps_needed + 7) / 8;
+    const int64_t max_blocks = static_cast<int64_t>(info.sm_count) * 8;
+    if (blocks > max_blocks) blocks = max_blocks;
+    if (blocks < 1) blocks = 1;
+    const uint16_t* x = reinterpret_cast<const uint16_t*>(d_x);
+    if (layout == NVFP4_SF_MMA)
+        quantize_kernel<true, kUnroll><<<static_cast<int>(blocks), 256, 0, stream>>>(
+            x, static_cast<int32_t>(M), static_cast<int32_t>(K), ld, d_g, segs, d_codes, d_sf,
+            static_cast<int32_t>(chunks), total);
+    else
+        quantize_kernel<false, kUnroll><<<static_cast<int>(blocks), 256, 0, stream>>>(
+            x, static_cast<int32_t>(M), static_cast<int32_t>(K), ld, d_g, segs, d_codes, d_sf,
+            static_cast<int32_t>(chunks), total);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+}
+
+nvfp4_status check_quantize_args(const void* d_x, int64_t rows, int64_t K, int64_t ld, const float* d_g,
+                                 const uint8_t* d_codes, const uint8_t* d_sf, nvfp4_sf_layout layout) {
+    if (d_x == nullptr || d_g == nullptr || d_codes == nullptr || d_sf == nullptr) return NVFP4_ERR_NULL;
+    if (rows < 0 || K <= 0 || (K % 16) != 0 || ld < K) return NVFP4_ERR_SHAPE;
+    if (layout != NVFP4_SF_LINEAR && layout != NVFP4_SF_MMA) return NVFP4_ERR_LAYOUT;
+    if (!aligned16(d_x) || (ld % 8) != 0 || !aligned16(d_codes)) return NVFP4_ERR_ALIGN;
+    if (layout == NVFP4_SF_MMA && (reinterpret_cast<uintptr_t>(d_sf) & 3u) != 0) return NVFP4_ERR_ALIGN;
+    return NVFP4_OK;
+}
+
+constexpr size_t kStatusBytes = 256;
+
+}  // namespace
+}  // namespace nvfp4
+
+using namespace nvfp4;
+
+extern "C" {
+
+size_t nvfp4_sf_bytes(int64_t rows, int64_t K, nvfp4_sf_layout layout) {
+    if (rows < 0 || K < 0 || (K % 16) != 0) return 0;
+    const int64_t kb = K / 16;
+    if (layout == NVFP4_SF_LINEAR) return static_cast<size_t>(rows * kb);
+    return static_cast<size_t>(((rows + 127) / 128) * ((kb + 3) / 4) * 512);
+}
+
+nvfp4_status nvfp4_calibrate(const void* d_x, int64_t rows, int64_t cols, int64_t ld, float* d_g, float* d_amax,
+                             void* stream) {
+    if (d_g == nullptr || (d_x == nullptr && rows * cols != 0)) return NVFP4_ERR_NULL;
+    if (rows < 0 || cols < 0 || ld < cols) return NVFP4_ERR_SHAPE;
+    DeviceInfo info;
+    nvfp4_status st = check_arch(info);
+    if (st != NVFP4_OK) return st;
+    cudaStream_t s = as_stream(stream);
+    if (cudaMemsetAsync(d_g, 0, sizeof(float), s) != cudaSuccess) return NVFP4_ERR_CUDA;
+    if (rows * cols > 0) {
+        const uint16_t* x = reinterpret_cast<const uint16_t*>(d_x);
+        const int64_t chunks = (cols + 255) / 256;
+        if (aligned16(d_x) && (ld % 8) == 0 && rows * chunks < (1ll << 31) && cols < (1ll << 31)) {
+            const int32_t total = static_cast<int32_t>(rows * chunks);
+            int64_t blocks = (total + 31) / 32;        // about four items per warp
+            const int64_t max_blocks = static_cast<int64_t>(info.sm_count) * 8;
+            if (blocks > max_blocks) blocks = max_blocks;
+            if (blocks < 1) blocks = 1;
+            amax_kernel<<<static_cast<int>(blocks), 256, 0, s>>>(x, static_cast<int32_t>(rows),
+                                                                 static_cast<int32_t>(cols), ld,
+                                                                 static_cast<int32_t>(chunks), total,
+                                                                 reinterpret_cast<uint32_t*>(d_g));
+        } else {
+            amax_scalar_kernel<<<info.sm_count * 4, 256, 0, s>>>(x, rows, cols, ld, reinterpret_cast<uint32_t*>(d_g));
+        }
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        if (cudaGetLastError() != cudaSuccess) return NVFP4_ERR_CUDA;
+    }
+    finalize_scale_kernel<<<1, 1, 0, s>>>(d_g, d_amax);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+}
+
+nvfp4_status nvfp4_quantize_act(const void* d_x, int64_t M, int64_t K, int64_t ld, const float* d_g,
+                                uint8_t* d_codes, uint8_t* d_sf, nvfp4_sf_layout layout, void* stream) {
+    nvfp4_status st = check_quantize_args(d_x, M, K, ld, d_g, d_codes, d_sf, layout);
+    if (st != NVFP4_OK) return st;
+    if (M == 0) return NVFP4_OK;
+    DeviceInfo info;
+    st = check_arch(info);
+    if (st != NVFP4_OK) return st;
+    SegTable segs;
+    std::memset(&segs, 0, sizeof(segs));
+    return quantize_impl(d_x, M, K, ld, d_g, segs, d_codes, d_sf, layout, info, as_stream(stream));
+}
+
+nvfp4_status nvfp4_quantize_weight(const void* d_w, int64_t N, int64_t K, int64_t ld, const nvfp4_segment* segs,
+                                   int nseg, float* d_g_seg, int calibrate_segments, uint8_t* d_codes,
+                                   uint8_t* d_sf, nvfp4_sf_layout layout, void* stream) {
+    nvfp4_status st = check_quantize_args(d_w, N, K, ld, d_g_seg, d_codes, d_sf, layout);
+    if (st != NVFP4_OK) return st;
+    st = check_segments(segs, nseg, N);
+    if (st != NVFP4_OK) return st;
+    if (N >= (1ll << 31)) return NVFP4_ERR_SHAPE;
+    DeviceInfo info;
+    st = check_arch(info);
+    if (st != NVFP4_OK) return st;
+    SegTable table;
+    std::memset(&table, 0, sizeof(table));
+    table.nseg = nseg;
+    for (int i = 0; i < nseg; ++i) table.row_end[i] = static_cast<int32_t>(segs[i].col_begin + segs[i].col_count);
+    if (calibrate_segments != 0) {
+        const uint16_t* w = reinterpret_cast<const uint16_t*>(d_w);
+        for (int i = 0; i < nseg; ++i) {
+            st = nvfp4_calibrate(w + segs[i].col_begin * ld, segs[i].col_count, K, ld, d_g_seg + i, nullptr, stream);
+            if (st != NVFP4_OK) return st;
+        }
+    }
+    return quantize_impl(d_w, N, K, ld, d_g_seg, table, d_codes, d_sf, layout, info, as_stream(stream));
+}
+
+size_t nvfp4_linear_workspace_bytes(int64_t, int64_t, int64_t, int) { return kStatusBytes; }
+
+nvfp4_status nvfp4_workspace_reset(void* d_workspace, size_t workspace_bytes, void* stream) {
+    if (d_workspace == nullptr) return NVFP4_ERR_NULL;
+    if (workspace_bytes < kStatusBytes) return NVFP4_ERR_WORKSPACE;
+    return cudaMemsetAsync(d_workspace, 0, kStatusBytes, as_stream(stream)) == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+}
+
+nvfp4_status nvfp4_linear(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const float* d_g_a, int64_t M,
+                          int64_t K, const uint8_t* d_w_codes, const uint8_t* d_w_sf, int64_t N,
+                          const nvfp4_segment* segs, const float* d_g_seg, int nseg, void* d_y, int64_t ldy,
+                          uint32_t flags, void* d_workspace, size_t workspace_bytes, void* stream) {
+    if (d_a_codes == nullptr || d_a_sf == nullptr || d_g_a == nullptr || d_w_codes == nullptr ||
+        d_w_sf == nullptr || d_g_seg == nullptr || d_y == nullptr)
+        return NVFP4_ERR_NULL;
+    if (M < 0 || N < 0 || K <= 0 || (K % 64) != 0 || ldy < N) return NVFP4_ERR_SHAPE;
+    if (M >= (1ll << 31) - 256 || N >= (1ll << 31) - 256 || K >= (1ll << 31)) return NVFP4_ERR_SHAPE;
+    nvfp4_status st = check_segments(segs, nseg, N);
+    if (N == 0 && segs != nullptr) st = NVFP4_OK;
+    if (st != NVFP4_OK) return st;
+    if (!aligned16(d_a_codes) || !aligned16(d_w_codes) || !aligned16(d_a_sf) || !aligned16(d_w_sf))
+        return NVFP4_ERR_ALIGN;
+    if (d_workspace == nullptr || workspace_bytes < kStatusBytes) return NVFP4_ERR_WORKSPACE;
+    if (!aligned16(d_workspace)) return NVFP4_ERR_ALIGN;
+    if ((flags & ~NVFP4_OUT_F32) != 0u) return NVFP4_ERR_SHAPE;
+    if (M == 0 || N == 0) return NVFP4_OK;
+    DeviceInfo info;
+    st = check_arch(info);
+    if (st != NVFP4_OK) return st;
+
+    const int bn = choose_variant(M, N);
+    CUtensorMap tmA, tmB;
+    st = codes_tensor_map(d_a_codes, M, K, kBM, &tmA);
+    if (st != NVFP4_OK) return st;
+    st = codes_tensor_map(d_w_codes, N, K, bn, &tmB);
+    if (st != NVFP4_OK) return st;
+
+    GemmParams p;
+    std::memset(&p, 0, sizeof(p));
+    p.sfa = d_a_sf;
+    p.sfb = d_w_sf;
+    p.g_a = d_g_a;
+    p.g_seg = d_g_seg;
+    p.y = d_y;
+    p.ldy = ldy;
+    p.status = reinterpret_cast<uint32_t*>(d_workspace);
+    p.M = static_cast<int32_t>(M);
+    p.N = static_cast<int32_t>(N);
+    p.K = static_cast<int32_t>(K);
+    p.m_tiles = static_cast<int32_t>((M + kBM - 1) / kBM);
+    p.k_tiles = static_cast<int32_t>((K + 255) / 256);
+    p.katoms = static_cast<int32_t>(K / 64);
+    p.sfa_bands = p.m_tiles;
+    p.sfb_bands = static_cast<int32_t>((N + 127) / 128);
+    p.flags = flags;
+    p.nseg = nseg;
+    for (int i = 0; i < nseg; ++i) p.seg_end[i] = static_cast<int32_t>(segs[i].col_begin + segs[i].col_count);
+    p.wait_limit_ns = kWaitLimitNs;
+    cudaStream_t s = as_stream(stream);
+    switch (bn) {
+        case 128: return launch_gemm<128, 2, 6>(tmA, tmB, p, info.sm_count, s);
+        case 256: return launch_gemm<256, 1, 4>(tmA, tmB, p, info.sm_count, s);
+        default: return NVFP4_ERR_SHAPE;
+    }
+}
+
+size_t nvfp4_linear_bf16_workspace_bytes(int64_t M, int64_t N, int64_t K, int nseg) {
+    (void)N; (void)nseg;
+    if (M < 0 || K < 0 || (K % 16) != 0) return 0;
+    const size_t codes = (static_cast<size_t>(M) * static_cast<size_t>(K / 2) + 255) & ~static_cast<size_t>(255);
+    return kStatusBytes + codes + nvfp4_sf_bytes(M, K, NVFP4_SF_MMA);
+}
+
+nvfp4_status nvfp4_linear_bf16(const void* d_x, int64_t ldx, const float* d_g_a, int64_t M, int64_t K,
+                               const uint8_t* d_w_codes, const uint8_t* d_w_sf, int64_t N,
+                               const nvfp4_segment* segs, const float* d_g_seg, int nseg, void* d_y, int64_t ldy,
+                               uint32_t flags, void* d_workspace, size_t workspace_bytes, void* stream) {
+    if (d_workspace == nullptr) return NVFP4_ERR_WORKSPACE;
+    if (M < 0 || K <= 0 || (K % 64) != 0) return NVFP4_ERR_SHAPE;
+    if (workspace_bytes < nvfp4_linear_bf16_workspace_bytes(M, N, K, nseg)) return NVFP4_ERR_WORKSPACE;
+    if (!aligned16(d_workspace)) return NVFP4_ERR_ALIGN;
+    uint8_t* ws = reinterpret_cast<uint8_t*>(d_workspace);
+    uint8_t* codes = ws + kStatusBytes;
+    const size_t codes_bytes = (static_cast<size_t>(M) * static_cast<size_t>(K / 2) + 255) & ~static_cast<size_t>(255);
+    uint8_t* sf = codes + codes_bytes;
+    nvfp4_status st = nvfp4_quantize_act(d_x, M, K, ldx, d_g_a, codes, sf, NVFP4_SF_MMA, stream);
+    if (st != NVFP4_OK) return st;
+    return nvfp4_linear(codes, sf, d_g_a, M, K, d_w_codes, d_w_sf, N, segs, d_g_seg, nseg, d_y, ldy, flags,
+                        d_workspace, kStatusBytes, stream);
+}
+
+nvfp4_status nvfp4_device_status(const void* d_workspace, void* stream) {
+    if (d_workspace == nullptr) return NVFP4_ERR_NULL;
+    uint32_t word = 0;
+    if (cudaMemcpyAsync(&word, d_workspace, sizeof(word), cudaMemcpyDeviceToHost, as_stream(stream)) != cudaSuccess)
+        return NVFP4_ERR_CUDA;
+    if (cudaStreamSynchronize(as_stream(stream)) != cudaSuccess) return NVFP4_ERR_CUDA;
+    return word == 0u ? NVFP4_OK : (word == NVFP4_ERR_TIMEOUT ? NVFP4_ERR_TIMEOUT : NVFP4_ERR_CUDA);
+}
+
+uint64_t nvfp4_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+nvfp4_status nvfp4_set_gemm_variant(int variant) {
+    if (variant != 0 && variant != 128 && variant != 256) return NVFP4_ERR_SHAPE;
+    g_variant.store(variant, std::memory_order_relaxed);
+    return NVFP4_OK;
+}
+
+const char* nvfp4_gemm_variants(void) { return "0=auto,128=128x128 tiles (2 accumulators),256=128x256 tiles"; }
+
+const char* nvfp4_status_string(nvfp4_status s) {
+    switch (s) {
+        case NVFP4_OK: return "ok";
+        case NVFP4_ERR_NULL: return "null pointer";
+        case NVFP4_ERR_SHAPE: return "bad shape or flag";
+        case NVFP4_ERR_ALIGN: return "misaligned pointer or leading dimension";
+        case NVFP4_ERR_SEGMENTS: return "segment table does not cover [0, N) in order";
+        case NVFP4_ERR_WORKSPACE: return "workspace missing or too small";
+        case NVFP4_ERR_ARCH: return "device is not compute capability 10.x";
+        case NVFP4_ERR_CUDA: return "CUDA call failed";
+        case NVFP4_ERR_TIMEOUT: return "a bounded in-kernel wait ran out";
+        case NVFP4_ERR_LAYOUT: return "unknown or unsupported scale layout";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

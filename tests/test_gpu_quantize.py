@@ -1,0 +1,124 @@
+"""GPU parity: calibrate / quantize_act / quantize_weight against the CPU oracle,
+bit-exact on packed codes and scale bytes, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2609_04098_b200 import binding as nv
+from paper_2609_04098_b200 import synth
+from tests import gpu_util as gu
+
+pytestmark = pytest.mark.gpu
+
+
+def _act_case(x_bits, g=None, layout=nv.SF_MMA, ld_pad=0):
+    M, K = x_bits.shape
+    xt = gu.dev_bf16(x_bits)
+    if ld_pad:
+        buf = torch.zeros((M, K + ld_pad), dtype=torch.bfloat16, device=gu.DEV)
+        buf[:, :K] = xt
+        xt = buf[:, :K]
+    if g is None:
+        amax_d = torch.zeros(1, dtype=torch.float32, device=gu.DEV)
+        g_d = nv.nvfp4_calibrate(xt, amax=amax_d)
+        amax_o, g_o = oracle.calibrate(x_bits)
+        assert amax_d.item() == amax_o and g_d.item() == g_o
+    else:
+        g_d = gu.dev_f32(g)
+        g_o = np.float32(g)
+    codes_d, sf_d = nv.nvfp4_quantize_act(xt, g_d, layout)
+    torch.cuda.synchronize()
+    codes_o, sf_o, _, _ = gu.oracle_quantized(x_bits, g=g_o)
+    gu.check_quantized(codes_d, sf_d, layout, codes_o, sf_o, K)
+    return codes_d, sf_d
+
+
+@pytest.mark.parametrize("layout", [nv.SF_MMA, nv.SF_LINEAR])
+def test_config1_activations(layout):
+    x, _, _ = synth.config1(0)
+    _act_case(x, layout=layout)
+
+
+@pytest.mark.parametrize("M,K", [(1, 16), (1, 5120), (3, 48), (16, 64), (17, 80), (127, 272), (129, 256),
+                                 (130, 1040), (257, 512), (300, 2064)])
+@pytest.mark.parametrize("layout", [nv.SF_MMA, nv.SF_LINEAR])
+def test_ragged_shapes(M, K, layout):
+    x = synth.config2_activations(7, M=M, K=K)
+    _act_case(x, layout=layout)
+
+
+def test_strided_input():
+    x = synth.prefill_activations(1, 3, 70, 320)
+    _act_case(x, ld_pad=24)
+
+
+def test_every_finite_bf16_pattern_at_several_scales():
+    # all 2^16 bit patterns minus NaN/Inf, laid out so that blocks mix magnitudes
+    pats = np.arange(65536, dtype=np.uint16)
+    finite = pats[(pats & 0x7F80) != 0x7F80]
+    rng = np.random.default_rng(0)
+    for g in (1.0, 0.37, 2.0 ** -20, 3.1e4):
+        x = rng.permutation(finite)[: (finite.size // 256) * 256].reshape(-1, 256)
+        _act_case(x, g=g)
+    # sorted order: neighbouring values share blocks, so codes span the whole grid incl. ties
+    x = finite[: (finite.size // 512) * 512].reshape(-1, 512)
+    _act_case(x, g=2.0 ** -3)
+    _act_case(x)
+
+
+def test_ties_zeros_signs_and_saturation():
+    vals = np.array([6.0, 0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0, -0.25, -0.75, -1.25, -1.75, -2.5, -3.5, -5.0, 0.0,
+                     0.0] * 1 + [-0.0] * 15 + [1e6, -1e6] + [1.0] * 14 + [1e-30, -1e-30] * 8)
+    x = synth.f64_to_bf16_bits(vals).reshape(1, 64)
+    _act_case(x, g=1.0)
+    _act_case(x, g=1e-3)        # static scale far too small: scale bytes and codes saturate
+    _act_case(np.zeros((5, 64), np.uint16))               # all-zero tensor: g = 1, everything 0
+    _act_case(np.full((5, 64), 0x8000, np.uint16))        # all -0
+
+
+def test_config2_full_size_bit_exact():
+    x = synth.config2_activations(0)
+    assert x.shape == (8192, 5120)
+    _act_case(x)
+
+
+def test_repeat_runs_are_identical():
+    x = synth.config2_activations(3, M=1024, K=5120)
+    xt = gu.dev_bf16(x)
+    g = nv.nvfp4_calibrate(xt)
+    c1, s1 = nv.nvfp4_quantize_act(xt, g)
+    c2, s2 = nv.nvfp4_quantize_act(xt, g)
+    torch.cuda.synchronize()
+    assert torch.equal(c1, c2) and torch.equal(s1, s2)
+
+
+@pytest.mark.parametrize("layout", [nv.SF_MMA, nv.SF_LINEAR])
+def test_weight_segments_calibrated_on_device(layout):
+    segs = synth.make_segments((("q", 64, 0.02), ("k", 40, 0.02), ("a", 48, 0.2), ("b", 9, 0.2)))
+    w = synth.weights(0, 5, segs, 320)
+    codes_d, sf_d, g_d = nv.nvfp4_quantize_weight(gu.dev_bf16(w), segs, None, layout)
+    torch.cuda.synchronize()
+    codes_o, sf_o, g_o, _ = gu.oracle_quantized(w, segments=segs)
+    assert np.array_equal(g_d.cpu().numpy(), g_o)
+    gu.check_quantized(codes_d, sf_d, layout, codes_o, sf_o, 320)
+
+
+def test_weight_segments_given_scales():
+    segs = synth.make_segments((("qkv", 96, 0.02), ("z", 96, 0.02)))
+    w = synth.weights(2, 5, segs, 256)
+    g_seg = np.float32([3.1e-5, 3.1e-5 / 1.82])
+    codes_d, sf_d, _ = nv.nvfp4_quantize_weight(gu.dev_bf16(w), segs, gu.dev_f32(g_seg), nv.SF_MMA)
+    torch.cuda.synchronize()
+    codes_o, sf_o, _, _ = gu.oracle_quantized(w, segments=segs, g_seg=g_seg)
+    gu.check_quantized(codes_d, sf_d, nv.SF_MMA, codes_o, sf_o, 256)
+
+
+def test_gdn_weight_full_size():
+    segs = synth.make_segments(synth.GDN_SEGMENTS)
+    w = synth.weights(0, 402, segs, synth.HIDDEN)
+    codes_d, sf_d, g_d = nv.nvfp4_quantize_weight(gu.dev_bf16(w), segs, None, nv.SF_MMA)
+    torch.cuda.synchronize()
+    codes_o, sf_o, g_o, _ = gu.oracle_quantized(w, segments=segs)
+    assert np.array_equal(g_d.cpu().numpy(), g_o)
+    gu.check_quantized(codes_d, sf_d, nv.SF_MMA, codes_o, sf_o, synth.HIDDEN)
