@@ -61,54 +61,62 @@ def ncu_traffic(name: str):
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
-              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-              "clocks_event_reasons.sw_power_cap")
+    """Samples SM clock and throttle reasons through NVML every few milliseconds while
+    the timed region runs (reading only; no setting is touched)."""
+    BITS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
 
-    def __init__(self, index: int):
-        self.rows = []
-        self.proc = None
-        self.index = index
+    def __init__(self, index: int, period_s: float = 0.004):
+        self.index, self.period = index, period_s
+        self.sm, self.power, self.reasons = [], [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self.thread = None
+        self.err = None
 
     def start(self):
         try:
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
-                 "--format=csv,noheader,nounits", "-lms", "100"],
-                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-            self.thread = threading.Thread(target=self._read, daemon=True)
-            self.thread.start()
-        except OSError:
-            self.proc = None
+            import pynvml
+            pynvml.nvmlInit()
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+            idx = self.index
+            if vis:
+                try:
+                    idx = int(vis.split(",")[self.index])
+                except ValueError:
+                    idx = self.index
+            h = pynvml.nvmlDeviceGetHandleByIndex(idx)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+        except Exception as e:                      # noqa: BLE001
+            self.err = "nvml unavailable: %s" % e
+            return
 
-    def _read(self):
-        for line in self.proc.stdout:
-            self.rows.append([c.strip() for c in line.split(",")])
+        def loop():
+            while not self._stop.is_set():
+                try:
+                    self.sm.append(float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)))
+                    self.power.append(pynvml.nvmlDeviceGetPowerUsage(h) / 1000.0)
+                    r = pynvml.nvmlDeviceGetCurrentClocksEventReasons(h)
+                    for bit, name in self.BITS.items():
+                        if r & bit:
+                            self.reasons.add(name)
+                except Exception as e:              # noqa: BLE001
+                    self.err = str(e)
+                    return
+                time.sleep(self.period)
+
+        self.thread = threading.Thread(target=loop, daemon=True)
+        self.thread.start()
 
     def stop(self):
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except subprocess.TimeoutExpired:
-            self.proc.kill()
-        sm, mx, reasons = [], [], set()
-        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
-        for r in self.rows:
-            if len(r) < 7:
-                continue
-            try:
-                sm.append(float(r[0]))
-                mx.append(float(r[1]))
-            except ValueError:
-                continue
-            for n, v in zip(names, r[3:7]):
-                if v.lower().startswith("active"):
-                    reasons.add(n)
-        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+        self._stop.set()
+        if self.thread is not None:
+            self.thread.join(timeout=2)
+        out = {"sm_mhz": float(np.median(self.sm)) if self.sm else None, "sm_max_mhz": self.max_mhz,
+               "sm_mhz_min": min(self.sm) if self.sm else None, "samples": len(self.sm),
+               "power_w_max": max(self.power) if self.power else None, "reasons": sorted(self.reasons)}
+        if self.err:
+            out["note"] = self.err
+        return out
 
 
 # --------------------------------------------------------------------------- workloads
@@ -303,6 +311,13 @@ def run_gpu(args):
         gemm_flops_per_launch = wl.flops / gemm_per_step
         achieved = gemm_flops_per_launch / (gemm_ms * 1e-3) / 1e12
         quant_in_step_gbs = wl.quant_elems / 2 * QUANT_BYTES_PER_ELEM / (quant_ms * 1e-3) / 1e9
+        gu_ms = span((gemm_slots[0],)) / args.steps
+        dn_ms = span((gemm_slots[1],)) / args.steps
+        result["gemm_detail"] = {
+            "gate_up": {"ms": round(gu_ms, 4), "tflops": round(gemm_flops(wl.M, 2 * INNER, HIDDEN) / gu_ms / 1e9, 1)},
+            "down": {"ms": round(dn_ms, 4), "tflops": round(gemm_flops(wl.M, HIDDEN, INNER) / dn_ms / 1e9, 1)},
+            "quantize_x1_us": round(span((quant_slots[0],)) / args.steps * 1e3, 2),
+            "quantize_x2_us": round(span((quant_slots[1],)) / args.steps * 1e3, 2)}
     else:
         gemm_ms = ms_per_step
         achieved = wl.flops / (gemm_ms * 1e-3) / 1e12
@@ -433,7 +448,8 @@ def cpu_baseline(wl, target_s=15.0, seed=0):
         return time.perf_counter() - t0
 
     t_small = run(8)
-    rows = int(max(8, min(1024, 8 * target_s / max(t_small, 1e-3))))
+    t_small = min(t_small, run(8))
+    rows = int(max(8, min(65536, 8 * target_s / max(t_small, 1e-4))))
     t = run(rows)
     flops = gemm_flops(rows, ncols, K)
     return {"value": round(flops / t / 1e12, 6), "unit": "TFLOP/s", "cores": oracle.num_threads(),
@@ -471,8 +487,8 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
-    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="mlp", choices=["mlp", "gdn", "linear"])
     ap.add_argument("--tokens", type=int, default=8192)

@@ -14,7 +14,7 @@ from typing import Optional, Sequence, Tuple
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libnvfp4_b200.so")
+LIB_PATH = os.environ.get("NVFP4_B200_LIB", os.path.join(_HERE, "libnvfp4_b200.so"))
 
 SF_LINEAR = 0
 SF_MMA = 1

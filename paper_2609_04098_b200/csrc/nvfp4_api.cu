@@ -3,6 +3,7 @@
 // no synchronisation (except nvfp4_device_status), nothing thrown.
 #include <atomic>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <unordered_map>
@@ -125,10 +126,38 @@ nvfp4_status codes_tensor_map(const uint8_t* d_codes, int64_t rows, int64_t K, i
     return NVFP4_OK;
 }
 
+// bf16 output [M, N] with row stride ldy, 32 x 64 boxes, 128-byte swizzle (TMA stores clip at M and N)
+nvfp4_status output_tensor_map(void* d_y, int64_t M, int64_t N, int64_t ldy, CUtensorMap* out) {
+    static std::mutex mu;
+    static std::unordered_map<MapKey, CUtensorMap, MapKeyHash> cache;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    MapKey key{d_y, M, N * 4096 + (ldy % 4096), static_cast<int>(ldy / 4096), dev};
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        auto it = cache.find(key);
+        if (it != cache.end()) { *out = it->second; return NVFP4_OK; }
+    }
+    EncodeTiledFn enc = encode_fn();
+    if (enc == nullptr) return NVFP4_ERR_CUDA;
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(N), static_cast<cuuint64_t>(M)};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(ldy) * 2u};
+    const cuuint32_t box[2] = {static_cast<cuuint32_t>(kOutPieceCols), 32u};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, d_y, dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return NVFP4_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (cache.size() > 4096) cache.clear();
+    cache[key] = *out;
+    return NVFP4_OK;
+}
+
 // ---------------------------------------------------------------- GEMM launch
 template <int BN, int ACC, int STAGES>
-nvfp4_status launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, GemmParams& p, int sm_count,
-                         cudaStream_t stream) {
+nvfp4_status launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY, GemmParams& p,
+                         int sm_count, cudaStream_t stream) {
     using C = GemmCfg<BN, ACC, STAGES>;
     static std::mutex mu;
     static std::unordered_map<int, bool> configured;
@@ -146,7 +175,7 @@ nvfp4_status launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, GemmPar
     p.n_tiles = (p.N + BN - 1) / BN;
     const int64_t tiles = static_cast<int64_t>(p.m_tiles) * p.n_tiles;
     const int grid = static_cast<int>(tiles < sm_count ? tiles : sm_count);
-    gemm_kernel<BN, ACC, STAGES><<<grid, kGemmThreads, C::SMEM_BYTES, stream>>>(tmA, tmB, p);
+    gemm_kernel<BN, ACC, STAGES><<<grid, kGemmThreads, C::SMEM_BYTES, stream>>>(tmA, tmB, tmY, p);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
@@ -326,6 +355,13 @@ nvfp4_status nvfp4_linear(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const
 
     GemmParams p;
     std::memset(&p, 0, sizeof(p));
+    CUtensorMap tmY;
+    std::memset(&tmY, 0, sizeof(tmY));
+    if ((flags & NVFP4_OUT_F32) == 0u && aligned16(d_y) && (ldy % 8) == 0) {
+        st = output_tensor_map(d_y, M, N, ldy, &tmY);
+        if (st != NVFP4_OK) return st;
+        p.tma_store = 1u;
+    }
     p.sfa = d_a_sf;
     p.sfb = d_w_sf;
     p.g_a = d_g_a;
@@ -345,10 +381,13 @@ nvfp4_status nvfp4_linear(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const
     p.nseg = nseg;
     for (int i = 0; i < nseg; ++i) p.seg_end[i] = static_cast<int32_t>(segs[i].col_begin + segs[i].col_count);
     p.wait_limit_ns = kWaitLimitNs;
+#ifdef NVFP4_PROBE
+    p.probe = getenv("NVFP4_PROBE") ? static_cast<uint32_t>(atoi(getenv("NVFP4_PROBE"))) : 0u;
+#endif
     cudaStream_t s = as_stream(stream);
     switch (bn) {
-        case 128: return launch_gemm<128, 2, 6>(tmA, tmB, p, info.sm_count, s);
-        case 256: return launch_gemm<256, 1, 4>(tmA, tmB, p, info.sm_count, s);
+        case 128: return launch_gemm<128, 2, 5>(tmA, tmB, tmY, p, info.sm_count, s);
+        case 256: return launch_gemm<256, 1, 3>(tmA, tmB, tmY, p, info.sm_count, s);
         default: return NVFP4_ERR_SHAPE;
     }
 }
