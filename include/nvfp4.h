@@ -177,9 +177,9 @@ nvfp4_status nvfp4_device_status(const void* d_workspace, void* stream);
 uint64_t nvfp4_launch_count(void);
 
 /*
- * Tile shape of the GEMM kernel: 0 = choose from the problem size (default),
- * otherwise one of the values nvfp4_status_string(NVFP4_OK)'s sibling
- * nvfp4_gemm_variants() lists.  Process-wide; meant for benchmarking.
+ * Tile shape of the GEMM kernel: 0 = choose from the problem size (default), otherwise
+ * one of the values that nvfp4_gemm_variants() lists ("value=description,...").
+ * Process-wide; meant for benchmarking and tests.  Errors: NVFP4_ERR_SHAPE.
  */
 nvfp4_status nvfp4_set_gemm_variant(int variant);
 const char* nvfp4_gemm_variants(void);

@@ -2,26 +2,32 @@
 //
 //   Y[m, n] = (sum_k a_hat[m,k] w_hat[n,k]) * g_a * g_seg[seg(n)]
 //
-// One persistent CTA per SM, 320 threads, four roles:
-//   warp 0      TMA producer: codes of A (128 x 256 elements) and W (BN x 256) per
-//               stage as 128-byte-swizzled tiles, plus their scale bytes, which are
-//               contiguous 512-byte atoms in the tensor-core scale layout and so
-//               travel as plain bulk copies;
-//   warps 6-9   scale loaders, one per 32-lane TMEM quarter: when a stage has landed
-//               they read its scale atoms from shared memory and write them into that
-//               stage's TMEM scale columns with tcgen05.st (a 512-byte atom is exactly
-//               32 lanes x 4 columns, identical in all four quarters).  tcgen05.cp could
-//               do this copy too, but it runs in the tensor pipe in series with the MMAs
-//               (measured: ~70 cycles each, three per 128-cycle MMA);
-//   warp 1      one thread walks the CTA's (tile, k) stream and issues tcgen05.mma
-//               kind::mxf4nvf4 (M=128, N=BN, K=64) into the TMEM accumulator as soon as
-//               a stage's scales are in TMEM;
-//   warps 2-5   epilogue: tcgen05.ld a 32-lane quarter each, multiply every column by
-//               its segment's global scale, round once to bf16, stage 32x64 pieces in
-//               swizzled shared memory and hand them to TMA stores; the accumulator
-//               is released as soon as its last column is in registers.
-// Stages hand over through mbarriers; every wait is bounded (see ptx.cuh) and a CTA
-// that gives up raises a status word instead of hanging.
+// One persistent CTA per SM (224 threads).  Two shapes of the same kernel:
+//   single  one CTA computes a 128 x BN tile (BN = 128 or 256);
+//   pair    two CTAs of a cluster compute a 256 x 256 tile with tcgen05 cta_group::2:
+//           each CTA loads 128 rows of A and only HALF of the W tile, so a stage is
+//           38 KB instead of 54 KB for the same tensor-core time and five stages fit.
+//           No load is multicast.  The partner's TMA copies count their bytes on the
+//           leader's "stage full" barrier; the leader's commits arrive on both CTAs'
+//           "stage empty" / "accumulator full" barriers; both CTAs' epilogue warps arrive
+//           on the leader's "accumulator empty" barrier.
+// Warp roles:
+//   warps 0-3   epilogue, one per 32-lane TMEM quarter: tcgen05.ld, multiply every column
+//               by its segment's global scale, round once to bf16, stage 32x64 pieces in
+//               swizzled shared memory, TMA store; the accumulator is handed back as soon
+//               as its last column is in registers;
+//   warp 4      TMA producer for A: codes (128 x 256 elements, 128-byte swizzle) and the
+//               matching scale atoms (a 3-D box over [band][k-atom][512 bytes]);
+//   warp 5      TMA producer for W, same;
+//   warp 6      one thread (leader CTA only, in a pair) issues, per K=64 step, the three
+//               tcgen05.cp that bring that step's scale atoms from shared memory to TMEM
+//               and then the tcgen05.mma kind::mxf4nvf4.  Measured on B200: an MMA of
+//               N=256 takes 128 cycles, a tcgen05.cp 64 cycles, and the copies run beside
+//               the MMAs, so the pipe settles at ~196 cycles per step.  (Moving the scales
+//               with ld.shared + tcgen05.st from other warps was tried: the loads starve
+//               behind the tensor core's own shared-memory reads.)
+// Every mbarrier wait is bounded (ptx.cuh); a CTA that gives up raises a status word and
+// tells its partner instead of hanging.
 #pragma once
 #include <cstdint>
 #include <cuda.h>
@@ -34,36 +40,40 @@
 namespace nvfp4 {
 
 struct GemmParams {
-    const uint8_t* sfa;      // A scales, tensor-core layout
-    const uint8_t* sfb;      // W scales, tensor-core layout
     const float* g_a;        // device scalar
     const float* g_seg;      // device [nseg]
     void* y;
     int64_t ldy;
     uint32_t* status;        // first word of the workspace
     int32_t M, N, K;
-    int32_t m_tiles, n_tiles, k_tiles;
+    int32_t m_tiles;         // ceil(M / 128)
+    int32_t n_tiles;         // ceil(N / BN)
+    int32_t k_tiles;         // ceil(K / 256)
     int32_t katoms;          // K / 64: 512-byte scale atoms per 128-row band
-    int32_t sfa_bands;       // ceil(M / 128)
-    int32_t sfb_bands;       // ceil(N / 128)
     uint32_t flags;
     uint32_t tma_store;      // 1: bf16 output through the TMA-store path (tmY valid)
     int32_t nseg;
     int32_t seg_end[NVFP4_MAX_SEGMENTS];
     uint64_t wait_limit_ns;
 #ifdef NVFP4_PROBE
-    uint32_t probe;          // timing experiments only (results are wrong): see the bits below
+    uint32_t probe;              // timing experiments only (results are wrong): see the bits below
+    unsigned long long* trace;   // [role][256] globaltimer stamps written by block 0
 #endif
 };
 #ifdef NVFP4_PROBE
 #define NVFP4_PROBE_BIT(p, b) (((p).probe >> (b)) & 1u)
+#define NVFP4_TRACE(p, role, idx)                                                        \
+    do {                                                                                 \
+        if ((p).trace != nullptr && blockIdx.x == 0 && (idx) < 256u)                     \
+            (p).trace[(role) * 256 + (idx)] = ptx::globaltimer_ns();                     \
+    } while (0)
 #else
 #define NVFP4_PROBE_BIT(p, b) 0u
+#define NVFP4_TRACE(p, role, idx) do {} while (0)
 #endif
-// probe bits: 0 no MMA, 1 no operand TMA, 2 no scale bulk copies, 3 no scale TMEM writes, 4 no epilogue
-// stores
+// probe bits: 0 no MMA, 1 no code loads, 2 no scale loads, 3 no scale copies to TMEM, 4 no epilogue stores
 
-constexpr int kGemmThreads = 320;
+constexpr int kGemmThreads = 224;
 constexpr int kBM = 128;
 constexpr int kBKBytes = 128;                 // 256 FP4 elements = one 128-byte swizzle row
 constexpr int kStepsPerStage = 4;             // four K=64 MMAs per stage
@@ -71,137 +81,138 @@ constexpr int kTmemCols = 512;
 constexpr int kOutPieceCols = 64;             // epilogue piece: 32 rows x 64 bf16 = 4 KB
 constexpr int kOutPieceBytes = 32 * kOutPieceCols * 2;
 
-template <int BN, int ACC, int STAGES>
+template <int BN, int STAGES, bool PAIR>
 struct GemmCfg {
+    static constexpr int ACC = (BN == 128) ? 2 : 1;                    // TMEM accumulators
+    static constexpr int B_ROWS = PAIR ? BN / 2 : BN;                  // W rows this CTA loads
+    static constexpr int NB_BANDS = BN / 128;                          // 128-row scale bands of the W tile
+    static constexpr int CTAS = PAIR ? 2 : 1;
     static constexpr int A_BYTES = kBM * kBKBytes;
-    static constexpr int B_BYTES = BN * kBKBytes;
-    static constexpr int NB_BANDS = BN / 128;
+    static constexpr int B_BYTES = B_ROWS * kBKBytes;
     static constexpr int SFA_BYTES = kStepsPerStage * 512;
     static constexpr int SFB_BYTES = NB_BANDS * kStepsPerStage * 512;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;
-    static constexpr int OUT_BYTES = 4 * 2 * kOutPieceBytes;          // per epilogue warp: two pieces
-    static constexpr int ALPHA_BYTES = 4 * BN * 4;                    // one private copy per epilogue warp
-    static constexpr int BAR_BYTES = (3 * STAGES + 2 * ACC + 1) * 8 + 16;
-    static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + OUT_BYTES + ALPHA_BYTES + BAR_BYTES;
+    static constexpr int OUT_BYTES = 4 * 2 * kOutPieceBytes;           // per epilogue warp: two pieces
+    static constexpr int BAR_BYTES = (2 * STAGES + 2 * ACC + 1) * 8 + 16;
+    static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + OUT_BYTES + BAR_BYTES;
     // TMEM columns: accumulators first, then one set of scale columns per smem stage
     static constexpr int SFA_SET_COLS = kStepsPerStage * 4;
     static constexpr int SFB_SET_COLS = kStepsPerStage * (BN / 32);
     static constexpr int SFA_COL0 = ACC * BN;
-    static constexpr int SFA_COLS = STAGES * SFA_SET_COLS;
-    static constexpr int SFB_COL0 = SFA_COL0 + SFA_COLS;
-    static constexpr int SFB_COLS = STAGES * SFB_SET_COLS;
-    static_assert(BN % 128 == 0 && BN <= 256, "BN must be 128 or 256");
-    static_assert(SFB_COL0 + SFB_COLS <= kTmemCols, "TMEM budget");
+    static constexpr int SFB_COL0 = SFA_COL0 + STAGES * SFA_SET_COLS;
+    static_assert(BN == 128 || BN == 256, "BN must be 128 or 256");
+    static_assert(!PAIR || BN == 256, "the pair kernel uses 256 x 256 tiles");
+    static_assert(SFB_COL0 + STAGES * SFB_SET_COLS <= kTmemCols, "TMEM budget");
     static_assert(SMEM_BYTES <= 232448, "shared memory budget");
     static_assert(STAGE_BYTES % 1024 == 0, "stage alignment");
 };
-
-// instruction descriptor: E2M1 x E2M1, E4M3 scales, K-major A and B, M=128, N=BN
-template <int BN>
-__device__ __forceinline__ constexpr uint32_t nvf4_idesc() {
-    return (1u << 7) | (1u << 10) | (static_cast<uint32_t>(BN >> 3) << 17) | (0u << 23) |
-           (static_cast<uint32_t>(kBM >> 4) << 24);
-}
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     __nv_bfloat162 b2 = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&b2);
 }
 
-template <int BN, int ACC, int STAGES>
+template <int BN, int STAGES, bool PAIR>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+            const __grid_constant__ CUtensorMap tmSFA, const __grid_constant__ CUtensorMap tmSFB,
             const __grid_constant__ CUtensorMap tmY, const __grid_constant__ GemmParams p) {
-    using C = GemmCfg<BN, ACC, STAGES>;
+    using C = GemmCfg<BN, STAGES, PAIR>;
+    constexpr int ACC = C::ACC;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* out_s = smem + STAGES * C::STAGE_BYTES;                   // 1024-byte aligned
-    float* alpha_s = reinterpret_cast<float*>(out_s + C::OUT_BYTES);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(out_s + C::OUT_BYTES + C::ALPHA_BYTES);
-    uint64_t* full = bars;
-    uint64_t* empty = bars + STAGES;
-    uint64_t* sfready = bars + 2 * STAGES;
-    uint64_t* tfull = bars + 3 * STAGES;
-    uint64_t* tempty = bars + 3 * STAGES + ACC;
-    uint64_t* drain = bars + 3 * STAGES + 2 * ACC;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(out_s + C::OUT_BYTES);
+    uint64_t* full = bars;                    // (leader's copy) every CTA's loads of a stage have landed
+    uint64_t* empty = bars + STAGES;          // the MMAs have finished reading a stage
+    uint64_t* tfull = bars + 2 * STAGES;      // accumulator complete
+    uint64_t* tempty = tfull + ACC;           // (leader's copy) every CTA has drained the accumulator
+    uint64_t* drain = tempty + ACC;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 1);
     volatile uint32_t* abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int32_t total_tiles = p.m_tiles * p.n_tiles;
-    const uint32_t my_tiles = (static_cast<uint32_t>(total_tiles) > blockIdx.x)
-                                  ? (static_cast<uint32_t>(total_tiles) - blockIdx.x + gridDim.x - 1) / gridDim.x
-                                  : 0u;
+    const uint32_t rank = PAIR ? ptx::cluster_ctarank() : 0u;          // 0 = leader
+    const uint32_t unit_id = PAIR ? (blockIdx.x >> 1) : blockIdx.x;    // CTA or cluster index
+    const uint32_t n_units = PAIR ? (gridDim.x >> 1) : gridDim.x;
+    const uint32_t m_units = PAIR ? (static_cast<uint32_t>(p.m_tiles) + 1u) >> 1 : static_cast<uint32_t>(p.m_tiles);
+    const uint32_t total_tiles = m_units * static_cast<uint32_t>(p.n_tiles);
+    const uint32_t my_tiles = total_tiles > unit_id ? (total_tiles - unit_id + n_units - 1) / n_units : 0u;
+    const uint32_t k_tiles = static_cast<uint32_t>(p.k_tiles);
+    const uint32_t total_it = my_tiles * k_tiles;
+    const uint32_t peer_abort =
+        PAIR ? ptx::mapa_shared(ptx::smem_u32(const_cast<uint32_t*>(abort_flag)), rank ^ 1u) : 0u;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            ptx::mbar_init(&full[s], 1);
+            ptx::mbar_init(&full[s], 2 * C::CTAS);       // the two producer threads of every CTA of the tile
             ptx::mbar_init(&empty[s], 1);
-            ptx::mbar_init(&sfready[s], 4);
         }
-        for (int a = 0; a < ACC; ++a) { ptx::mbar_init(&tfull[a], 1); ptx::mbar_init(&tempty[a], 4); }
+        for (int a = 0; a < ACC; ++a) {
+            ptx::mbar_init(&tfull[a], 1);
+            ptx::mbar_init(&tempty[a], 4 * C::CTAS);     // epilogue warps of every CTA of the tile
+        }
         ptx::mbar_init(drain, 1);
         *abort_flag = 0u;
         ptx::fence_barrier_init();
     }
-    // scale staging starts as zeros so that bands a tile never loads read as 0.0, not NaN
-    for (int s = 0; s < STAGES; ++s) {
-        uint4* z = reinterpret_cast<uint4*>(smem + s * C::STAGE_BYTES + C::A_BYTES + C::B_BYTES);
-        for (int i = threadIdx.x; i < (C::SFA_BYTES + C::SFB_BYTES) / 16; i += kGemmThreads)
-            z[i] = make_uint4(0u, 0u, 0u, 0u);
-    }
-    ptx::fence_proxy_async_smem();
-    if (warp == 1) {
-        ptx::tmem_alloc(tmem_slot, kTmemCols);
-        ptx::tmem_relinquish();
+    if (warp == 6) {
+        if (PAIR) { ptx::tmem_alloc_pair(tmem_slot, kTmemCols); ptx::tmem_relinquish_pair(); }
+        else      { ptx::tmem_alloc(tmem_slot, kTmemCols);      ptx::tmem_relinquish(); }
     }
     ptx::tc_fence_before();
-    __syncthreads();
+    if (PAIR) ptx::cluster_sync_all(); else __syncthreads();   // barriers and TMEM exist from here on
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer
+    // tile index -> (row unit, column tile); row units vary fastest so that the CTAs running
+    // at the same time share W tiles through L2
+    auto tile_of = [&](uint32_t t, int32_t& um, int32_t& un) {
+        const uint32_t tile = unit_id + t * n_units;
+        um = static_cast<int32_t>(tile % m_units);
+        un = static_cast<int32_t>(tile / m_units);
+    };
+
+    if (warp == 4 || warp == 5) {
+        // ------------------------------------------------------------ TMA producers
         if (lane == 0) {
-            ptx::prefetch_tensormap(&tmA);
-            ptx::prefetch_tensormap(&tmB);
+            const bool is_a = warp == 4;
+            const uint32_t leader_full = PAIR ? ptx::mapa_shared(ptx::smem_u32(full), 0u) : 0u;
+            const CUtensorMap* tm_codes = is_a ? &tmA : &tmB;
+            const CUtensorMap* tm_sf = is_a ? &tmSFA : &tmSFB;
+            ptx::prefetch_tensormap(tm_codes);
+            ptx::prefetch_tensormap(tm_sf);
+            const uint32_t code_off = is_a ? 0u : C::A_BYTES;
+            const uint32_t sf_off = C::A_BYTES + C::B_BYTES + (is_a ? 0u : C::SFA_BYTES);
+            uint32_t tx = is_a ? (C::A_BYTES + C::SFA_BYTES) : (C::B_BYTES + C::SFB_BYTES);
+#ifdef NVFP4_PROBE
+            if (NVFP4_PROBE_BIT(p, 1)) tx -= is_a ? C::A_BYTES : C::B_BYTES;
+            if (NVFP4_PROBE_BIT(p, 2)) tx -= is_a ? C::SFA_BYTES : C::SFB_BYTES;
+#endif
             uint32_t it = 0;
             bool ok = true;
-            for (int32_t tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-                const int32_t m_t = tile % p.m_tiles, n_t = tile / p.m_tiles;
+            for (uint32_t t = 0; ok && t < my_tiles; ++t) {
+                int32_t um, un;
+                tile_of(t, um, un);
+                const int32_t a_band = PAIR ? 2 * um + static_cast<int32_t>(rank) : um;
+                const int32_t code_row = is_a ? a_band * kBM : un * BN + static_cast<int32_t>(rank) * C::B_ROWS;
+                const int32_t sf_band = is_a ? a_band : un * C::NB_BANDS;
                 for (int32_t kt = 0; kt < p.k_tiles; ++kt, ++it) {
                     const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-                    if (!ptx::mbar_wait_bounded(&empty[s], ph ^ 1u, abort_flag, p.wait_limit_ns)) { ok = false; break; }
+                    if (!ptx::mbar_wait_bounded(&empty[s], ph ^ 1u, abort_flag, p.wait_limit_ns, peer_abort)) { ok = false; break; }
+                    if (is_a) NVFP4_TRACE(p, 0, it);
                     uint8_t* st = smem + s * C::STAGE_BYTES;
-                    const int32_t steps = min(kStepsPerStage, p.katoms - kt * kStepsPerStage);
-                    const uint32_t sf_bytes = static_cast<uint32_t>(steps) * 512u;
-                    uint32_t tx = C::A_BYTES + C::B_BYTES + sf_bytes;
-                    int nb_live = 0;
-#pragma unroll
-                    for (int c = 0; c < C::NB_BANDS; ++c)
-                        if (n_t * C::NB_BANDS + c < p.sfb_bands) ++nb_live;
-                    tx += nb_live * sf_bytes;
-#ifdef NVFP4_PROBE
-                    if (NVFP4_PROBE_BIT(p, 1)) tx -= C::A_BYTES + C::B_BYTES;
-                    if (NVFP4_PROBE_BIT(p, 2)) tx -= (1 + nb_live) * sf_bytes;
-#endif
-                    ptx::mbar_arrive_expect_tx(&full[s], tx);
-                    if (!NVFP4_PROBE_BIT(p, 1)) {
-                        ptx::tma_load_2d(st, &tmA, kt * kBKBytes, m_t * kBM, &full[s]);
-                        ptx::tma_load_2d(st + C::A_BYTES, &tmB, kt * kBKBytes, n_t * BN, &full[s]);
-                    }
-                    if (NVFP4_PROBE_BIT(p, 2)) continue;
-                    ptx::bulk_load(st + C::A_BYTES + C::B_BYTES,
-                                   p.sfa + (static_cast<int64_t>(m_t) * p.katoms + kt * kStepsPerStage) * 512,
-                                   sf_bytes, &full[s]);
-#pragma unroll
-                    for (int c = 0; c < C::NB_BANDS; ++c) {
-                        const int32_t band = n_t * C::NB_BANDS + c;
-                        if (band < p.sfb_bands)
-                            ptx::bulk_load(st + C::A_BYTES + C::B_BYTES + C::SFA_BYTES + c * (kStepsPerStage * 512),
-                                           p.sfb + (static_cast<int64_t>(band) * p.katoms + kt * kStepsPerStage) * 512,
-                                           sf_bytes, &full[s]);
+                    // rows / bands / k-atoms past the tensor are zero-filled by TMA
+                    if (PAIR) {
+                        const uint32_t bar = leader_full + s * 8u;
+                        ptx::mbar_arrive_expect_tx_cluster(bar, tx);
+                        if (!NVFP4_PROBE_BIT(p, 1)) ptx::tma_load_2d_pair(st + code_off, tm_codes, kt * kBKBytes, code_row, bar);
+                        if (!NVFP4_PROBE_BIT(p, 2)) ptx::tma_load_3d_pair(st + sf_off, tm_sf, 0, kt * kStepsPerStage, sf_band, bar);
+                    } else {
+                        ptx::mbar_arrive_expect_tx(&full[s], tx);
+                        if (!NVFP4_PROBE_BIT(p, 1)) ptx::tma_load_2d(st + code_off, tm_codes, kt * kBKBytes, code_row, &full[s]);
+                        if (!NVFP4_PROBE_BIT(p, 2)) ptx::tma_load_3d(st + sf_off, tm_sf, 0, kt * kStepsPerStage, sf_band, &full[s]);
                     }
                 }
             }
@@ -212,179 +223,191 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     for (int spin = 0; spin < 4096 && !ptx::mbar_try_wait(&full[i % STAGES], (i / STAGES) & 1u); ++spin) {}
             }
         }
-    } else if (warp == 1) {
+    } else if (warp == 6) {
         // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc = nvf4_idesc<BN>();
-            const uint32_t k_tiles = static_cast<uint32_t>(p.k_tiles);
-            const uint32_t total_it = my_tiles * k_tiles;
+        // The tensor pipe accepts only about one instruction ahead of the one it is executing, so
+        // the instruction stream between two MMAs has to be short: the ring of stages is unrolled
+        // (every shared-memory and TMEM address is base + compile-time constant), descriptors are
+        // a fixed high word and an incremented low word, there are no divisions, and the next
+        // stage's barrier is polled before the current stage's last MMA.  The whole warp walks
+        // the loop so that all of this stays warp-uniform (tcgen05 operands are uniform
+        // registers; computed under a single-lane branch they cost a vector->uniform move chain
+        // per issue); one elected lane, the same throughout, issues.
+        if (rank == 0) {
+            const bool leader = ptx::elect_one();
+            // E2M1 x E2M1, E4M3 scales, K-major A and B; M = 128 (single) or 256 (pair), N = BN
+            constexpr uint32_t idesc = (1u << 7) | (1u << 10) | (static_cast<uint32_t>(BN >> 3) << 17) |
+                                       (static_cast<uint32_t>((PAIR ? 256 : 128) >> 4) << 24);
+            // descriptor words (see ptx::smem_desc): codes use the 128-byte swizzle with 1024 bytes
+            // between 8-row groups; scale atoms are unswizzled with 128 bytes between 8-row groups
+            constexpr uint32_t kCodeHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+            constexpr uint32_t kCodeLoFlags = (16u >> 4) << 16;
+            constexpr uint32_t kScaleHi = (128u >> 4) | (1u << 14);
+            const uint32_t smem_enc = (ptx::smem_u32(smem) & 0x3FFFFu) >> 4;      // stage 0, in 16-byte units
+            auto desc = [](uint32_t lo, uint32_t hi) { return (static_cast<uint64_t>(hi) << 32) | lo; };
+            const int32_t tail_steps = p.katoms - (p.k_tiles - 1) * kStepsPerStage;   // K-steps of a tile's last stage
             bool ok = true;
-            for (uint32_t it = 0; ok && it < total_it; ++it) {
-                const uint32_t kt = it % k_tiles, tl = it / k_tiles;
-                const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-                const uint32_t acc = tl % ACC, aph = (tl / ACC) & 1u;
-                if (NVFP4_PROBE_BIT(p, 0)) {
-                    if (!ptx::mbar_wait_bounded(&sfready[s], ph, abort_flag, p.wait_limit_ns)) { ok = false; break; }
-                    ptx::mbar_arrive(&empty[s]);
-                    if (kt == k_tiles - 1) {
-                        if (!ptx::mbar_wait_bounded(&tempty[acc], aph ^ 1u, abort_flag, p.wait_limit_ns)) { ok = false; break; }
-                        ptx::mbar_arrive(&tfull[acc]);
+            uint32_t it = 0, kt = 0, acc = 0, aph = 0, ph = 0;
+            bool have_full = false;          // the coming iteration's "stage full" was already observed
+            while (ok && it < total_it) {
+#pragma unroll
+                for (int s = 0; s < STAGES; ++s) {
+                    if (it >= total_it) break;
+                    if (kt == 0) {
+                        if (!ptx::mbar_wait_bounded(&tempty[acc], aph ^ 1u, abort_flag, p.wait_limit_ns, peer_abort)) { ok = false; break; }
+                        if (have_full) ptx::tc_fence_after();
                     }
-                    continue;
+                    if (!have_full) {
+                        if (!ptx::mbar_wait_bounded(&full[s], ph, abort_flag, p.wait_limit_ns, peer_abort)) { ok = false; break; }
+                        ptx::tc_fence_after();
+                    }
+                    have_full = false;
+                    if (leader) NVFP4_TRACE(p, 2, it);
+                    const uint32_t st_enc = smem_enc + s * (C::STAGE_BYTES >> 4);
+                    const uint32_t sfa_t = tmem_base + C::SFA_COL0 + s * C::SFA_SET_COLS;
+                    const uint32_t sfb_t = tmem_base + C::SFB_COL0 + s * C::SFB_SET_COLS;
+                    const uint32_t d_tmem = tmem_base + acc * BN;
+                    const bool last_kt = kt + 1 == k_tiles;
+                    const int32_t steps = last_kt ? tail_steps : kStepsPerStage;
+#pragma unroll
+                    for (int j = 0; j < kStepsPerStage; ++j) {
+                        if (j < steps) {
+                            if (j == kStepsPerStage - 1 && it + 1 < total_it) {
+                                // while the earlier steps run: has the next stage landed?
+                                const int ns = (s + 1 == STAGES) ? 0 : s + 1;
+                                if (ptx::mbar_try_wait(&full[ns], ns == 0 ? ph ^ 1u : ph)) { ptx::tc_fence_after(); have_full = true; }
+                            }
+                            // this step's scale atoms: shared -> TMEM (32 rows x 16 bytes each, replicated into
+                            // the four lane quarters), then the MMA that reads them
+                            if (!NVFP4_PROBE_BIT(p, 3) && leader) {
+                                const uint32_t sf_enc = st_enc + ((C::A_BYTES + C::B_BYTES + j * 512) >> 4);
+                                if (PAIR) {
+                                    ptx::tc_cp_32x128b_warpx4_pair(sfa_t + j * 4, desc(sf_enc, kScaleHi));
+                                    ptx::tc_cp_32x128b_warpx4_pair(sfb_t + j * (BN / 32), desc(sf_enc + (C::SFA_BYTES >> 4), kScaleHi));
+                                    if (C::NB_BANDS == 2)
+                                        ptx::tc_cp_32x128b_warpx4_pair(sfb_t + j * (BN / 32) + 4,
+                                                                       desc(sf_enc + ((C::SFA_BYTES + kStepsPerStage * 512) >> 4), kScaleHi));
+                                } else {
+                                    ptx::tc_cp_32x128b_warpx4(sfa_t + j * 4, desc(sf_enc, kScaleHi));
+                                    ptx::tc_cp_32x128b_warpx4(sfb_t + j * (BN / 32), desc(sf_enc + (C::SFA_BYTES >> 4), kScaleHi));
+                                    if (C::NB_BANDS == 2)
+                                        ptx::tc_cp_32x128b_warpx4(sfb_t + j * (BN / 32) + 4,
+                                                                  desc(sf_enc + ((C::SFA_BYTES + kStepsPerStage * 512) >> 4), kScaleHi));
+                                }
+                            }
+                            if (!NVFP4_PROBE_BIT(p, 0) && leader) {
+                                // advancing K by 64 elements = 32 bytes inside the 128-byte swizzle row
+                                const uint64_t a_desc = desc((st_enc + j * 2) | kCodeLoFlags, kCodeHi);
+                                const uint64_t b_desc = desc((st_enc + (C::A_BYTES >> 4) + j * 2) | kCodeLoFlags, kCodeHi);
+                                const uint32_t accum = (j == 0) ? (kt != 0u ? 1u : 0u) : 1u;
+                                if (PAIR) ptx::tc_mma_nvf4_pair(d_tmem, a_desc, b_desc, idesc, sfa_t + j * 4, sfb_t + j * (BN / 32), accum);
+                                else      ptx::tc_mma_nvf4(d_tmem, a_desc, b_desc, idesc, sfa_t + j * 4, sfb_t + j * (BN / 32), accum);
+                            }
+                        }
+                    }
+                    // stage reusable once these MMAs have read it; after the last K tile the accumulator is complete
+                    if (leader) {
+                        if (PAIR) {
+                            ptx::tc_commit_pair(&empty[s], 3);
+                            if (last_kt) ptx::tc_commit_pair(&tfull[acc], 3);
+                        } else {
+                            ptx::tc_commit(&empty[s]);
+                            if (last_kt) ptx::tc_commit(&tfull[acc]);
+                        }
+                        NVFP4_TRACE(p, 3, it);
+                    }
+                    ++it;
+                    if (last_kt) {
+                        kt = 0;
+                        if (ACC == 1) { aph ^= 1u; } else { acc ^= 1u; if (acc == 0u) aph ^= 1u; }
+                    } else {
+                        ++kt;
+                    }
                 }
-                if (kt == 0) {
-                    if (!ptx::mbar_wait_bounded(&tempty[acc], aph ^ 1u, abort_flag, p.wait_limit_ns)) { ok = false; break; }
-                }
-                // scales in TMEM implies codes in shared memory (the loaders waited for the stage)
-                if (!ptx::mbar_wait_bounded(&sfready[s], ph, abort_flag, p.wait_limit_ns)) { ok = false; break; }
-                ptx::tc_fence_after();
-                const uint32_t st = ptx::smem_u32(smem + s * C::STAGE_BYTES);
-                const int32_t steps = min(kStepsPerStage, p.katoms - static_cast<int32_t>(kt) * kStepsPerStage);
-                const uint32_t sfa_t = tmem_base + C::SFA_COL0 + s * C::SFA_SET_COLS;
-                const uint32_t sfb_t = tmem_base + C::SFB_COL0 + s * C::SFB_SET_COLS;
-                const uint32_t d_tmem = tmem_base + acc * BN;
-                const uint64_t a_desc = ptx::smem_desc(st, 16, 1024, 2);
-                const uint64_t b_desc = ptx::smem_desc(st + C::A_BYTES, 16, 1024, 2);
-                for (int32_t j = 0; j < steps; ++j) {
-                    // advancing K by 64 elements = 32 bytes inside the 128-byte swizzle row
-                    ptx::tc_mma_nvf4(d_tmem, a_desc + 2u * j, b_desc + 2u * j, idesc, sfa_t + j * 4,
-                                     sfb_t + j * (BN / 32), (kt | static_cast<uint32_t>(j)) != 0u ? 1u : 0u);
-                }
-                ptx::tc_commit(&empty[s]);                          // stage reusable once these MMAs have read it
-                if (kt == k_tiles - 1) ptx::tc_commit(&tfull[acc]); // accumulator complete
+                ph ^= 1u;
             }
             if (!ok) {
-                ptx::tc_commit(drain);                  // let issued MMAs finish before TMEM is freed
+                // let issued MMAs finish before TMEM is freed
+                if (leader) { if (PAIR) ptx::tc_commit_pair(drain, 1); else ptx::tc_commit(drain); }
                 for (int spin = 0; spin < (1 << 16) && !ptx::mbar_try_wait(drain, 0u); ++spin) {}
             }
         }
-    } else if (warp >= 6) {
-        // ------------------------------------------------------------ scale loaders
-        // A stage's TMEM scale columns are free when its shared-memory buffers are: the
-        // producer refilled the stage only after the MMAs that read both had completed.
-        const uint32_t quarter = static_cast<uint32_t>(warp & 3);
-        const uint32_t k_tiles = static_cast<uint32_t>(p.k_tiles);
-        const uint32_t total_it = my_tiles * k_tiles;
-        const uint32_t lane_field = (quarter * 32u) << 16;
-        for (uint32_t it = 0; it < total_it; ++it) {
-            const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-            bool ok = ptx::mbar_wait_bounded(&full[s], ph, abort_flag, p.wait_limit_ns);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            if (!NVFP4_PROBE_BIT(p, 3)) {
-                const uint32_t sf_s = ptx::smem_u32(smem + s * C::STAGE_BYTES) + C::A_BYTES + C::B_BYTES + lane * 16;
-                // A: atom j -> columns 4j..4j+3
-                {
-                    uint32_t r[16];
-#pragma unroll
-                    for (int j = 0; j < kStepsPerStage; ++j) {
-                        const uint4 v = ptx::ld_shared_v4(sf_s + j * 512);
-                        r[4 * j + 0] = v.x; r[4 * j + 1] = v.y; r[4 * j + 2] = v.z; r[4 * j + 3] = v.w;
-                    }
-                    ptx::tmem_st_32x16(tmem_base + lane_field + C::SFA_COL0 + s * C::SFA_SET_COLS, r);
-                }
-                // W: K-step j, 128-row band c -> columns j*(BN/32) + 4c ..
-#pragma unroll
-                for (int c = 0; c < C::NB_BANDS; ++c) {
-                    uint32_t r[16];
-#pragma unroll
-                    for (int j = 0; j < kStepsPerStage; ++j) {
-                        const uint4 v = ptx::ld_shared_v4(sf_s + C::SFA_BYTES + c * (kStepsPerStage * 512) + j * 512);
-                        r[4 * j + 0] = v.x; r[4 * j + 1] = v.y; r[4 * j + 2] = v.z; r[4 * j + 3] = v.w;
-                    }
-                    if (C::NB_BANDS == 1) {
-                        ptx::tmem_st_32x16(tmem_base + lane_field + C::SFB_COL0 + s * C::SFB_SET_COLS, r);
-                    } else {
-                        // bands interleave per K-step: four columns at a time
-#pragma unroll
-                        for (int j = 0; j < kStepsPerStage; ++j) {
-                            const uint32_t q[4] = {r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]};
-                            ptx::tmem_st_32x4(tmem_base + lane_field + C::SFB_COL0 + s * C::SFB_SET_COLS +
-                                              j * (BN / 32) + c * 4, q);
-                        }
-                    }
-                }
-                ptx::tmem_st_wait();
-            }
-            ptx::tc_fence_before();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(&sfready[s]);
-        }
-    } else {
+    } else if (warp < 4) {
         // ------------------------------------------------------------ epilogue
-        const int quarter = warp & 3;                   // TMEM lanes this warp may read
-        float* alpha_w = alpha_s + quarter * BN;
+        const int quarter = warp;                       // TMEM lanes this warp may read
         uint8_t* out_w = out_s + quarter * (2 * kOutPieceBytes);
         const float g_a = __ldg(p.g_a);
         const bool out_f32 = (p.flags & NVFP4_OUT_F32) != 0u;
         const bool use_tma = p.tma_store != 0u;
-        const bool vec_ok = out_f32 ? ((p.ldy & 3) == 0 && (reinterpret_cast<uintptr_t>(p.y) & 15) == 0)
-                                    : ((p.ldy & 7) == 0 && (reinterpret_cast<uintptr_t>(p.y) & 15) == 0);
+        const uint32_t leader_tempty = PAIR ? ptx::mapa_shared(ptx::smem_u32(tempty), 0u) : ptx::smem_u32(tempty);
         if (use_tma && lane == 0) ptx::prefetch_tensormap(&tmY);
-        uint32_t tl = 0, pieces_stored = 0;
-        for (int32_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++tl) {
-            const int32_t m_t = tile % p.m_tiles, n_t = tile / p.m_tiles;
-            const int32_t n0 = n_t * BN;
-            const uint32_t acc = tl % ACC, aph = (tl / ACC) & 1u;
-            // per-column global scale of this tile (each warp keeps a private copy)
-            __syncwarp();
-            for (int c = lane; c < BN; c += 32) {
-                const int32_t n = n0 + c;
+        uint32_t pieces_stored = 0;
+        for (uint32_t t = 0; t < my_tiles; ++t) {
+            int32_t um, un;
+            tile_of(t, um, un);
+            const int32_t n0 = un * BN;
+            const uint32_t acc = t % ACC, aph = (t / ACC) & 1u;
+            if (warp == 0 && lane == 0) NVFP4_TRACE(p, 7, t);
+            // global scale of columns n0 + 32 i + lane, i = 0 .. BN/32-1, in registers
+            float areg[BN / 32];
+#pragma unroll
+            for (int i = 0; i < BN / 32; ++i) {
+                const int32_t n = n0 + i * 32 + lane;
                 float a = 0.0f;
                 if (n < p.N) {
                     int sgi = 0;
                     while (sgi + 1 < p.nseg && n >= p.seg_end[sgi]) ++sgi;
                     a = __fmul_rn(g_a, __ldg(p.g_seg + sgi));
                 }
-                alpha_w[c] = a;
+                areg[i] = a;
             }
-            __syncwarp();
-            bool ok = ptx::mbar_wait_bounded(&tfull[acc], aph, abort_flag, p.wait_limit_ns);
-            ok = __all_sync(0xffffffffu, ok);
+            // one lane polls, with a back-off: 128 threads spinning on the barrier would take
+            // shared-memory cycles away from the MMAs for the whole main loop
+            bool ok = true;
+            if (lane == 0) ok = ptx::mbar_wait_bounded(&tfull[acc], aph, abort_flag, p.wait_limit_ns, peer_abort, 128u);
+            ok = __shfl_sync(0xffffffffu, static_cast<int>(ok), 0) != 0;
             if (!ok) break;
             ptx::tc_fence_after();
+            if (warp == 0 && lane == 0) NVFP4_TRACE(p, 6, t);
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * BN;
-            const int32_t row0 = m_t * kBM + quarter * 32;
-
-            if (use_tma) {
-                constexpr int NP = BN / kOutPieceCols;
-                uint32_t ra[64], rb[64];
-                ptx::tmem_ld_32x64(t_row, ra);
+            const int32_t row0 = (PAIR ? 2 * um + static_cast<int32_t>(rank) : um) * kBM + quarter * 32;
+            constexpr int NP = BN / kOutPieceCols;
+            uint32_t ra[64], rb[64];
+            ptx::tmem_ld_32x64(t_row, ra);
 #pragma unroll
-                for (int pc = 0; pc < NP; ++pc) {
-                    uint32_t (&cur)[64] = (pc & 1) ? rb : ra;
-                    uint32_t (&nxt)[64] = (pc & 1) ? ra : rb;
-                    ptx::tmem_ld_wait();
-                    if (pc + 1 < NP) {
-                        ptx::tmem_ld_32x64(t_row + (pc + 1) * kOutPieceCols, nxt);
-                    } else {
-                        // last column is in registers: hand the accumulator back to the MMA warp
-                        ptx::tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive(&tempty[acc]);
+            for (int pc = 0; pc < NP; ++pc) {
+                uint32_t (&cur)[64] = (pc & 1) ? rb : ra;
+                uint32_t (&nxt)[64] = (pc & 1) ? ra : rb;
+                ptx::tmem_ld_wait();
+                if (pc + 1 < NP) {
+                    ptx::tmem_ld_32x64(t_row + (pc + 1) * kOutPieceCols, nxt);
+                } else {
+                    // last column is in registers: hand the accumulator back to the MMA issuer
+                    ptx::tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) {
+                        if (PAIR) ptx::mbar_arrive_cluster(leader_tempty + acc * 8u);
+                        else      ptx::mbar_arrive(&tempty[acc]);
                     }
-                    const int32_t col0 = n0 + pc * kOutPieceCols;
-                    if (col0 >= p.N || row0 >= p.M || NVFP4_PROBE_BIT(p, 4)) continue;   // warp-uniform
+                }
+                const int32_t col0 = n0 + pc * kOutPieceCols;
+                if (col0 >= p.N || row0 >= p.M || NVFP4_PROBE_BIT(p, 4)) continue;        // warp-uniform
+                float v[64];
+#pragma unroll
+                for (int j = 0; j < 64; ++j)
+                    v[j] = __fmul_rn(__uint_as_float(cur[j]), __shfl_sync(0xffffffffu, areg[pc * 2 + (j >> 5)], j & 31));
+                if (use_tma) {
                     uint8_t* buf = out_w + (pieces_stored & 1u) * kOutPieceBytes;
                     if (pieces_stored >= 2u) {
                         if (lane == 0) ptx::bulk_wait_group_read<1>();   // the store that last used `buf` has read it
                         __syncwarp();
                     }
-                    const float* al = alpha_w + pc * kOutPieceCols;
                     const uint32_t row_s = ptx::smem_u32(buf) + lane * 128;
 #pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        const uint32_t w0 = pack_bf16x2(__fmul_rn(__uint_as_float(cur[8 * c + 0]), al[8 * c + 0]),
-                                                        __fmul_rn(__uint_as_float(cur[8 * c + 1]), al[8 * c + 1]));
-                        const uint32_t w1 = pack_bf16x2(__fmul_rn(__uint_as_float(cur[8 * c + 2]), al[8 * c + 2]),
-                                                        __fmul_rn(__uint_as_float(cur[8 * c + 3]), al[8 * c + 3]));
-                        const uint32_t w2 = pack_bf16x2(__fmul_rn(__uint_as_float(cur[8 * c + 4]), al[8 * c + 4]),
-                                                        __fmul_rn(__uint_as_float(cur[8 * c + 5]), al[8 * c + 5]));
-                        const uint32_t w3 = pack_bf16x2(__fmul_rn(__uint_as_float(cur[8 * c + 6]), al[8 * c + 6]),
-                                                        __fmul_rn(__uint_as_float(cur[8 * c + 7]), al[8 * c + 7]));
-                        // 128-byte swizzle: 16-byte chunk index XOR (row mod 8)
-                        ptx::st_shared_v4(row_s + ((c ^ (lane & 7)) << 4), w0, w1, w2, w3);
-                    }
+                    for (int c = 0; c < 8; ++c)     // 128-byte swizzle: 16-byte chunk index XOR (row mod 8)
+                        ptx::st_shared_v4(row_s + ((c ^ (lane & 7)) << 4), pack_bf16x2(v[8 * c + 0], v[8 * c + 1]),
+                                          pack_bf16x2(v[8 * c + 2], v[8 * c + 3]), pack_bf16x2(v[8 * c + 4], v[8 * c + 5]),
+                                          pack_bf16x2(v[8 * c + 6], v[8 * c + 7]));
                     ptx::fence_proxy_async_smem();
                     __syncwarp();
                     if (lane == 0) {
@@ -392,60 +415,22 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                         ptx::bulk_commit_group();
                     }
                     ++pieces_stored;
-                }
-            } else {
-                const int32_t row = row0 + lane;
-                const bool row_ok = row < p.M;
-#pragma unroll 1
-                for (int c = 0; c < BN / 32; ++c) {
-                    uint32_t r[32];
-                    __syncwarp();
-                    ptx::tmem_ld_32x32(t_row + c * 32, r);
-                    ptx::tmem_ld_wait();
-                    const int32_t col0 = n0 + c * 32;
-                    if (!row_ok || col0 >= p.N || NVFP4_PROBE_BIT(p, 4)) continue;
-                    const float* al = alpha_w + c * 32;
-                    if (out_f32) {
-                        float* yr = reinterpret_cast<float*>(p.y) + static_cast<int64_t>(row) * p.ldy + col0;
+                } else {
+                    // plain stores: float32 output, or bf16 rows that TMA cannot address
+                    const int32_t row = row0 + lane;
+                    if (row < p.M) {
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            float4 o;
-                            o.x = __fmul_rn(__uint_as_float(r[4 * j + 0]), al[4 * j + 0]);
-                            o.y = __fmul_rn(__uint_as_float(r[4 * j + 1]), al[4 * j + 1]);
-                            o.z = __fmul_rn(__uint_as_float(r[4 * j + 2]), al[4 * j + 2]);
-                            o.w = __fmul_rn(__uint_as_float(r[4 * j + 3]), al[4 * j + 3]);
-                            if (vec_ok && col0 + 4 * j + 4 <= p.N) {
-                                *reinterpret_cast<float4*>(yr + 4 * j) = o;
-                            } else {
-                                const float e[4] = {o.x, o.y, o.z, o.w};
-                                for (int t = 0; t < 4; ++t)
-                                    if (col0 + 4 * j + t < p.N) yr[4 * j + t] = e[t];
-                            }
-                        }
-                    } else {
-                        __nv_bfloat16* yr =
-                            reinterpret_cast<__nv_bfloat16*>(p.y) + static_cast<int64_t>(row) * p.ldy + col0;
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            uint32_t w[4];
-#pragma unroll
-                            for (int t = 0; t < 4; ++t)
-                                w[t] = pack_bf16x2(__fmul_rn(__uint_as_float(r[8 * j + 2 * t]), al[8 * j + 2 * t]),
-                                                   __fmul_rn(__uint_as_float(r[8 * j + 2 * t + 1]), al[8 * j + 2 * t + 1]));
-                            if (vec_ok && col0 + 8 * j + 8 <= p.N) {
-                                *reinterpret_cast<uint4*>(yr + 8 * j) = make_uint4(w[0], w[1], w[2], w[3]);
-                            } else {
-                                for (int t = 0; t < 8; ++t)
-                                    if (col0 + 8 * j + t < p.N)
-                                        reinterpret_cast<uint16_t*>(yr)[8 * j + t] =
-                                            static_cast<uint16_t>((t & 1) ? (w[t >> 1] >> 16) : (w[t >> 1] & 0xFFFFu));
+                        for (int j = 0; j < 64; ++j) {
+                            if (col0 + j < p.N) {
+                                if (out_f32)
+                                    reinterpret_cast<float*>(p.y)[static_cast<int64_t>(row) * p.ldy + col0 + j] = v[j];
+                                else
+                                    reinterpret_cast<__nv_bfloat16*>(p.y)[static_cast<int64_t>(row) * p.ldy + col0 + j] =
+                                        __float2bfloat16_rn(v[j]);
                             }
                         }
                     }
                 }
-                ptx::tc_fence_before();
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(&tempty[acc]);
             }
         }
         if (use_tma && lane == 0) ptx::bulk_wait_group<0>();   // all output stores complete before exit
@@ -453,10 +438,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 
     // ---------------------------------------------------------------- teardown
     ptx::tc_fence_before();
-    __syncthreads();
-    if (warp == 1) {
+    if (PAIR) ptx::cluster_sync_all(); else __syncthreads();   // nobody touches TMEM or a partner's barriers after this
+    if (warp == 6) {
         ptx::tc_fence_after();
-        ptx::tmem_dealloc(tmem_base, kTmemCols);
+        if (PAIR) ptx::tmem_dealloc_pair(tmem_base, kTmemCols); else ptx::tmem_dealloc(tmem_base, kTmemCols);
     }
     if (threadIdx.x == 0 && *abort_flag != 0u) atomicExch(p.status, static_cast<uint32_t>(NVFP4_ERR_TIMEOUT));
 }

@@ -126,6 +126,36 @@ nvfp4_status codes_tensor_map(const uint8_t* d_codes, int64_t rows, int64_t K, i
     return NVFP4_OK;
 }
 
+// scale bytes in the tensor-core layout seen as [band][k-atom][128 x u32]; a box takes four
+// k-atoms of `box_bands` bands; bands and k-atoms past the tensor read as zero
+nvfp4_status scales_tensor_map(const uint8_t* d_sf, int64_t rows, int64_t K, int box_bands, CUtensorMap* out) {
+    static std::mutex mu;
+    static std::unordered_map<MapKey, CUtensorMap, MapKeyHash> cache;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const int64_t bands = (rows + 127) / 128, katoms = K / 64;
+    MapKey key{d_sf, bands, katoms, box_bands, dev};
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        auto it = cache.find(key);
+        if (it != cache.end()) { *out = it->second; return NVFP4_OK; }
+    }
+    EncodeTiledFn enc = encode_fn();
+    if (enc == nullptr) return NVFP4_ERR_CUDA;
+    const cuuint64_t dims[3] = {128, static_cast<cuuint64_t>(katoms), static_cast<cuuint64_t>(bands)};
+    const cuuint64_t strides[2] = {512, static_cast<cuuint64_t>(katoms) * 512u};
+    const cuuint32_t box[3] = {128, static_cast<cuuint32_t>(kStepsPerStage), static_cast<cuuint32_t>(box_bands)};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<uint8_t*>(d_sf), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return NVFP4_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (cache.size() > 4096) cache.clear();
+    cache[key] = *out;
+    return NVFP4_OK;
+}
+
 // bf16 output [M, N] with row stride ldy, 32 x 64 boxes, 128-byte swizzle (TMA stores clip at M and N)
 nvfp4_status output_tensor_map(void* d_y, int64_t M, int64_t N, int64_t ldy, CUtensorMap* out) {
     static std::mutex mu;
@@ -155,35 +185,65 @@ nvfp4_status output_tensor_map(void* d_y, int64_t M, int64_t N, int64_t ldy, CUt
 }
 
 // ---------------------------------------------------------------- GEMM launch
-template <int BN, int ACC, int STAGES>
-nvfp4_status launch_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY, GemmParams& p,
-                         int sm_count, cudaStream_t stream) {
-    using C = GemmCfg<BN, ACC, STAGES>;
+struct GemmMaps {
+    CUtensorMap a, b, sfa, sfb, y;
+};
+
+template <int BN, int STAGES, bool PAIR>
+nvfp4_status launch_gemm(const GemmMaps& tm, GemmParams& p, int sm_count, cudaStream_t stream) {
+    using C = GemmCfg<BN, STAGES, PAIR>;
     static std::mutex mu;
-    static std::unordered_map<int, bool> configured;
+    static std::unordered_map<int, int> max_units;      // per device: CTAs (single) or clusters (pair); 0 = unset
     int dev = 0;
     cudaGetDevice(&dev);
+    p.n_tiles = (p.N + BN - 1) / BN;
+    const int64_t m_units = PAIR ? (p.m_tiles + 1) / 2 : p.m_tiles;
+    const int64_t tiles = m_units * p.n_tiles;
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof(cfg));
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = PAIR ? 2 : 1;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.blockDim = dim3(kGemmThreads, 1, 1);
+    cfg.dynamicSmemBytes = C::SMEM_BYTES;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int units = 0;
     {
         std::lock_guard<std::mutex> lock(mu);
-        if (!configured[dev]) {
-            if (cudaFuncSetAttribute(gemm_kernel<BN, ACC, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        units = max_units[dev];
+        if (units == 0) {
+            if (cudaFuncSetAttribute(gemm_kernel<BN, STAGES, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      C::SMEM_BYTES) != cudaSuccess)
                 return NVFP4_ERR_CUDA;
-            configured[dev] = true;
+            units = PAIR ? sm_count / 2 : sm_count;
+            if (PAIR) {
+                cfg.gridDim = dim3(static_cast<unsigned>(sm_count & ~1), 1, 1);
+                int n = 0;
+                if (cudaOccupancyMaxActiveClusters(&n, gemm_kernel<BN, STAGES, PAIR>, &cfg) == cudaSuccess && n >= 1) {
+                    if (n < units) units = n;
+                } else {
+                    cudaGetLastError();
+                }
+            }
+            max_units[dev] = units;
         }
     }
-    p.n_tiles = (p.N + BN - 1) / BN;
-    const int64_t tiles = static_cast<int64_t>(p.m_tiles) * p.n_tiles;
-    const int grid = static_cast<int>(tiles < sm_count ? tiles : sm_count);
-    gemm_kernel<BN, ACC, STAGES><<<grid, kGemmThreads, C::SMEM_BYTES, stream>>>(tmA, tmB, tmY, p);
+    const int64_t use = tiles < units ? tiles : units;
+    cfg.gridDim = dim3(static_cast<unsigned>((PAIR ? 2 : 1) * use), 1, 1);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, gemm_kernel<BN, STAGES, PAIR>, tm.a, tm.b, tm.sfa, tm.sfb, tm.y, p);
     g_launches.fetch_add(1, std::memory_order_relaxed);
-    return cudaGetLastError() == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+    return e == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
 
+// 128 / 256: one CTA per 128 x BN tile; 2: CTA pair per 256 x 256 tile
 int choose_variant(int64_t M, int64_t N) {
     const int forced = g_variant.load(std::memory_order_relaxed);
     if (forced != 0) return forced;
-    (void)M;
+    if (M > 128 && N >= 256) return 2;
     return N >= 256 ? 256 : 128;
 }
 
@@ -347,23 +407,25 @@ nvfp4_status nvfp4_linear(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const
     if (st != NVFP4_OK) return st;
 
     const int bn = choose_variant(M, N);
-    CUtensorMap tmA, tmB;
-    st = codes_tensor_map(d_a_codes, M, K, kBM, &tmA);
+    const int tile_n = bn == 128 ? 128 : 256;
+    GemmMaps tm;
+    std::memset(&tm, 0, sizeof(tm));
+    st = codes_tensor_map(d_a_codes, M, K, kBM, &tm.a);
     if (st != NVFP4_OK) return st;
-    st = codes_tensor_map(d_w_codes, N, K, bn, &tmB);
+    st = codes_tensor_map(d_w_codes, N, K, bn == 2 ? 128 : tile_n, &tm.b);
+    if (st != NVFP4_OK) return st;
+    st = scales_tensor_map(d_a_sf, M, K, 1, &tm.sfa);
+    if (st != NVFP4_OK) return st;
+    st = scales_tensor_map(d_w_sf, N, K, tile_n / 128, &tm.sfb);
     if (st != NVFP4_OK) return st;
 
     GemmParams p;
     std::memset(&p, 0, sizeof(p));
-    CUtensorMap tmY;
-    std::memset(&tmY, 0, sizeof(tmY));
     if ((flags & NVFP4_OUT_F32) == 0u && aligned16(d_y) && (ldy % 8) == 0) {
-        st = output_tensor_map(d_y, M, N, ldy, &tmY);
+        st = output_tensor_map(d_y, M, N, ldy, &tm.y);
         if (st != NVFP4_OK) return st;
         p.tma_store = 1u;
     }
-    p.sfa = d_a_sf;
-    p.sfb = d_w_sf;
     p.g_a = d_g_a;
     p.g_seg = d_g_seg;
     p.y = d_y;
@@ -375,19 +437,19 @@ nvfp4_status nvfp4_linear(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const
     p.m_tiles = static_cast<int32_t>((M + kBM - 1) / kBM);
     p.k_tiles = static_cast<int32_t>((K + 255) / 256);
     p.katoms = static_cast<int32_t>(K / 64);
-    p.sfa_bands = p.m_tiles;
-    p.sfb_bands = static_cast<int32_t>((N + 127) / 128);
     p.flags = flags;
     p.nseg = nseg;
     for (int i = 0; i < nseg; ++i) p.seg_end[i] = static_cast<int32_t>(segs[i].col_begin + segs[i].col_count);
     p.wait_limit_ns = kWaitLimitNs;
 #ifdef NVFP4_PROBE
     p.probe = getenv("NVFP4_PROBE") ? static_cast<uint32_t>(atoi(getenv("NVFP4_PROBE"))) : 0u;
+    p.trace = getenv("NVFP4_TRACE_PTR") ? reinterpret_cast<unsigned long long*>(strtoull(getenv("NVFP4_TRACE_PTR"), nullptr, 16)) : nullptr;
 #endif
     cudaStream_t s = as_stream(stream);
     switch (bn) {
-        case 128: return launch_gemm<128, 2, 5>(tmA, tmB, tmY, p, info.sm_count, s);
-        case 256: return launch_gemm<256, 1, 3>(tmA, tmB, tmY, p, info.sm_count, s);
+        case 128: return launch_gemm<128, 5, false>(tm, p, info.sm_count, s);
+        case 256: return launch_gemm<256, 3, false>(tm, p, info.sm_count, s);
+        case 2: return launch_gemm<256, 5, true>(tm, p, info.sm_count, s);
         default: return NVFP4_ERR_SHAPE;
     }
 }
@@ -429,12 +491,14 @@ nvfp4_status nvfp4_device_status(const void* d_workspace, void* stream) {
 uint64_t nvfp4_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 nvfp4_status nvfp4_set_gemm_variant(int variant) {
-    if (variant != 0 && variant != 128 && variant != 256) return NVFP4_ERR_SHAPE;
+    if (variant != 0 && variant != 128 && variant != 256 && variant != 2) return NVFP4_ERR_SHAPE;
     g_variant.store(variant, std::memory_order_relaxed);
     return NVFP4_OK;
 }
 
-const char* nvfp4_gemm_variants(void) { return "0=auto,128=128x128 tiles (2 accumulators),256=128x256 tiles"; }
+const char* nvfp4_gemm_variants(void) {
+    return "0=auto,128=128x128 tiles (2 accumulators),256=128x256 tiles,2=256x256 tiles on CTA pairs";
+}
 
 const char* nvfp4_status_string(nvfp4_status s) {
     switch (s) {

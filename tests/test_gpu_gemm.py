@@ -12,7 +12,7 @@ from tests import gpu_util as gu
 
 pytestmark = pytest.mark.gpu
 
-VARIANTS = [128, 256]
+VARIANTS = [128, 256, 2]
 
 
 @pytest.fixture(autouse=True)
