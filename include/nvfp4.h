@@ -93,7 +93,7 @@ nvfp4_status nvfp4_calibrate(const void* d_x, int64_t rows, int64_t cols, int64_
  * fused multiply-add:
  *     s8   = e4m3_rne_sat( bmax * (1 / (6 * g)) )
  *     code = e2m1_rne_sat( x * (1 / (e4m3(s8) * g)) )     (all codes 0 if s8 == 0)
- *   d_x      bf16 [M, K], row stride ld elements; 16-byte aligned, ld % 8 == 0
+ *   d_x      bf16 [M, K], row stride ld elements; 32-byte aligned, ld % 16 == 0 (256-bit loads)
  *   d_g      in: the tensor's global scale (device scalar)
  *   d_codes  out: [M, K/2] bytes, 16-byte aligned
  *   d_sf     out: nvfp4_sf_bytes(M, K, layout) bytes (padding is written as zero)
@@ -149,7 +149,7 @@ size_t nvfp4_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int nseg);
  * The same layer fed with bf16 activations: quantization runs inside the call
  * (paper: Section 9, "Decode overhead" -- activation quantization is the overhead
  * that matters at small batch), codes and scales live in the workspace.
- *   d_x   bf16 [M, K], row stride ldx, 16-byte aligned, ldx % 8 == 0
+ *   d_x   bf16 [M, K], row stride ldx, 32-byte aligned, ldx % 16 == 0
  */
 nvfp4_status nvfp4_linear_bf16(const void* d_x, int64_t ldx, const float* d_g_a,
                                int64_t M, int64_t K,

@@ -250,8 +250,8 @@ int choose_variant(int64_t M, int64_t N) {
 nvfp4_status quantize_impl(const void* d_x, int64_t M, int64_t K, int64_t ld, const float* d_g,
                            const SegTable& segs, uint8_t* d_codes, uint8_t* d_sf, nvfp4_sf_layout layout,
                            const DeviceInfo& info, cudaStream_t stream) {
-    const int64_t chunks = (K + 255) / 256;
-    if (M * chunks >= (1ll << 31) || K >= (1ll << 31)) return NVFP4_ERR_SHAPE;
+    const int64_t chunks = (K + 511) / 512;              // 512 elements = one block per lane
+    if (M >= (1ll << 31) || K >= (1ll << 31)) return NVFP4_ERR_SHAPE;
     if (layout == NVFP4_SF_MMA && (M % 128) != 0) {
         // rows of the last 128-row band that the tensor does not have must read as zero scales
         const int64_t katoms = (K / 16 + 3) / 4;
@@ -259,22 +259,28 @@ nvfp4_status quantize_impl(const void* d_x, int64_t M, int64_t K, int64_t ld, co
             cudaSuccess)
             return NVFP4_ERR_CUDA;
     }
-    const int32_t total = static_cast<int32_t>(M * chunks);
-    constexpr int kUnroll = 4;
-    const int64_t warps_needed = (total + kUnroll - 1) / kUnroll;
-    int64_t blocks = (warps_needed + 7) / 8;
-    const int64_t max_blocks = static_cast<int64_t>(info.sm_count) * 8;
+    // a unit = up to `per_unit` consecutive chunks of one row; units per row rounded up to a power of two
+    constexpr int kUnroll = 2;
+    const int64_t resident_warps = static_cast<int64_t>(info.sm_count) * 48;
+    int64_t per_unit = (M * chunks > 2 * resident_warps) ? kUnroll : 1;
+    int split_log2 = 0;
+    while ((1ll << split_log2) * per_unit < chunks) ++split_log2;
+    per_unit = (chunks + (1ll << split_log2) - 1) >> split_log2;
+    const int64_t units = M << split_log2;
+    if (units >= (1ll << 31)) return NVFP4_ERR_SHAPE;
+    int64_t blocks = (units + 7) / 8;
+    const int64_t max_blocks = static_cast<int64_t>(info.sm_count) * 6;
     if (blocks > max_blocks) blocks = max_blocks;
     if (blocks < 1) blocks = 1;
     const uint16_t* x = reinterpret_cast<const uint16_t*>(d_x);
     if (layout == NVFP4_SF_MMA)
         quantize_kernel<true, kUnroll><<<static_cast<int>(blocks), 256, 0, stream>>>(
             x, static_cast<int32_t>(M), static_cast<int32_t>(K), ld, d_g, segs, d_codes, d_sf,
-            static_cast<int32_t>(chunks), total);
+            static_cast<int32_t>(chunks), static_cast<int32_t>(per_unit), split_log2, static_cast<int32_t>(units));
     else
         quantize_kernel<false, kUnroll><<<static_cast<int>(blocks), 256, 0, stream>>>(
             x, static_cast<int32_t>(M), static_cast<int32_t>(K), ld, d_g, segs, d_codes, d_sf,
-            static_cast<int32_t>(chunks), total);
+            static_cast<int32_t>(chunks), static_cast<int32_t>(per_unit), split_log2, static_cast<int32_t>(units));
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
@@ -284,7 +290,7 @@ nvfp4_status check_quantize_args(const void* d_x, int64_t rows, int64_t K, int64
     if (d_x == nullptr || d_g == nullptr || d_codes == nullptr || d_sf == nullptr) return NVFP4_ERR_NULL;
     if (rows < 0 || K <= 0 || (K % 16) != 0 || ld < K) return NVFP4_ERR_SHAPE;
     if (layout != NVFP4_SF_LINEAR && layout != NVFP4_SF_MMA) return NVFP4_ERR_LAYOUT;
-    if (!aligned16(d_x) || (ld % 8) != 0 || !aligned16(d_codes)) return NVFP4_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(d_x) & 31u) != 0 || (ld % 16) != 0 || !aligned16(d_codes)) return NVFP4_ERR_ALIGN;
     if (layout == NVFP4_SF_MMA && (reinterpret_cast<uintptr_t>(d_sf) & 3u) != 0) return NVFP4_ERR_ALIGN;
     return NVFP4_OK;
 }

@@ -1,13 +1,15 @@
 // Bandwidth-bound kernels: per-tensor amax (calibration) and bf16 -> NVFP4
 // quantization (E2M1 codes + one E4M3 scale per 16 elements).
 //
-// Work decomposition: one warp owns 256 consecutive elements of one row (one
-// 128-bit load per lane, fully coalesced 512 bytes per warp).  Two neighbouring
-// lanes hold one 16-element block, so the block maximum is one shuffle; eight
-// lanes hold the four blocks whose scale bytes form one 32-bit word of the
-// tensor-core scale layout.
+// Work decomposition: one lane owns one 16-element block (a 256-bit load; a warp reads
+// 1024 contiguous bytes), so the block maximum needs no shuffle and there is one reciprocal
+// per 16 elements; four neighbouring lanes hold the four scale bytes that form one 32-bit
+// word of the tensor-core scale layout.  The kernel is issue-bound before it is
+// bandwidth-bound, so the instruction count per element is what was optimised: packed
+// bf16 maximum, no per-item division, per-row constants hoisted.
 #pragma once
 #include <cstdint>
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
 #include "../../include/nvfp4.h"
@@ -66,75 +68,120 @@ __device__ __forceinline__ int64_t sf_mma_offset(int32_t r, int32_t b, int32_t k
     return (static_cast<int64_t>(r >> 7) * katoms + (b >> 2)) * 512 + (rr & 31) * 16 + (rr >> 5) * 4 + (b & 3);
 }
 
-// One 8-element slice of a block: returns the packed codes, and the block's scale
-// byte through s8_out.  The operation order is the contract the bit-exact
-// comparison relies on (binary32, RNE, no fused multiply-add).
-__device__ __forceinline__ uint32_t quantize_slice(const float (&f)[8], float g, float c1, uint32_t& s8_out) {
-    float m = fmaxf(fmaxf(fmaxf(fabsf(f[0]), fabsf(f[1])), fmaxf(fabsf(f[2]), fabsf(f[3]))),
-                    fmaxf(fmaxf(fabsf(f[4]), fabsf(f[5])), fmaxf(fabsf(f[6]), fabsf(f[7]))));
-    m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));          // the other half of the block
-    const uint32_t s8 = f32_to_e4m3(__fmul_rn(m, c1));
-    s8_out = s8;
-    if (s8 == 0u) return 0u;
-    const float d = __fmul_rn(e4m3_to_f32(s8), g);
-    const float q = __fdiv_rn(1.0f, d);
-    float y[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) y[i] = __fmul_rn(f[i], q);
-    return f32x8_to_e2m1(y);
+// 256-bit streaming load: one 16-element block (32 bytes of bf16) per lane, never reused
+__device__ __forceinline__ void ldg256_stream(const void* p, uint32_t (&v)[8]) {
+    asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+                 : "l"(p));
 }
 
+__device__ __forceinline__ uint32_t bf16x2_absmax(uint32_t a, uint32_t b) {
+    __nv_bfloat162 r = __hmax2(*reinterpret_cast<__nv_bfloat162*>(&a), *reinterpret_cast<__nv_bfloat162*>(&b));
+    return *reinterpret_cast<uint32_t*>(&r);
+}
+
+// One 16-element block held by one lane: returns the 16 packed codes (element i in nibble i)
+// and the block's scale byte.  The operation order is the contract the bit-exact comparison
+// relies on (binary32, round-to-nearest-even, no fused multiply-add):
+//     s8 = e4m3(bmax * c1),  c1 = 1 / (6 g);   code = e2m1(x * (1 / (e4m3(s8) * g)))
+__device__ __forceinline__ uint2 quantize_block(const uint32_t (&v)[8], float g, float c1, uint32_t& s8_out) {
+    // block maximum on packed bf16 pairs (|x| is a bit mask; the maximum of bf16 values is exact)
+    uint32_t m = bf16x2_absmax(v[0] & 0x7FFF7FFFu, v[1] & 0x7FFF7FFFu);
+    m = bf16x2_absmax(m, bf16x2_absmax(v[2] & 0x7FFF7FFFu, v[3] & 0x7FFF7FFFu));
+    uint32_t m2 = bf16x2_absmax(v[4] & 0x7FFF7FFFu, v[5] & 0x7FFF7FFFu);
+    m2 = bf16x2_absmax(m2, bf16x2_absmax(v[6] & 0x7FFF7FFFu, v[7] & 0x7FFF7FFFu));
+    m = bf16x2_absmax(m, m2);
+    const float bmax = fmaxf(__uint_as_float(m << 16), __uint_as_float(m & 0xFFFF0000u));
+    const uint32_t s8 = f32_to_e4m3(__fmul_rn(bmax, c1));
+    s8_out = s8;
+    const float d = __fmul_rn(e4m3_to_f32(s8), g);
+    const float q = __fdiv_rn(1.0f, d);                       // s8 == 0 gives inf; that block is zeroed below
+    uint2 out;
+    {
+        float y[8];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            y[2 * i] = __fmul_rn(__uint_as_float(v[i] << 16), q);
+            y[2 * i + 1] = __fmul_rn(__uint_as_float(v[i] & 0xFFFF0000u), q);
+        }
+        out.x = f32x8_to_e2m1(y);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            y[2 * i] = __fmul_rn(__uint_as_float(v[4 + i] << 16), q);
+            y[2 * i + 1] = __fmul_rn(__uint_as_float(v[4 + i] & 0xFFFF0000u), q);
+        }
+        out.y = f32x8_to_e2m1(y);
+    }
+    if (s8 == 0u) out = make_uint2(0u, 0u);                   // scale rounds to zero: codes 0, signs cleared
+    return out;
+}
+
+// A warp owns `chunks_per_unit` consecutive 512-element chunks of one row (a "unit"); units are
+// dealt round-robin to a persistent grid.  split_log2: log2 of the units per row.
 template <bool MMA_LAYOUT, int UNROLL>
 __global__ void __launch_bounds__(256)
 quantize_kernel(const uint16_t* __restrict__ x, int32_t M, int32_t K, int64_t ld,
                 const float* __restrict__ g_ptr, SegTable segs,
                 uint8_t* __restrict__ codes, uint8_t* __restrict__ sf,
-                int32_t chunks_per_row, int32_t total_items) {
+                int32_t chunks_per_row, int32_t chunks_per_unit, int32_t split_log2, int32_t total_units) {
     const int lane = threadIdx.x & 31;
     const int32_t warp_global = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int32_t nwarps = gridDim.x * (blockDim.x >> 5);
     const int32_t KB = K >> 4;
     const int32_t katoms = (KB + 3) >> 2;
     const float g_single = (segs.nseg == 0) ? __ldg(g_ptr) : 0.0f;
+    const float c1_single = __fdiv_rn(1.0f, __fmul_rn(6.0f, g_single));
 
-    for (int32_t base = warp_global; base < total_items; base += nwarps * UNROLL) {
-        uint4 v[UNROLL];
-        int32_t row[UNROLL], col[UNROLL];
-        bool live[UNROLL];
-#pragma unroll
-        for (int u = 0; u < UNROLL; ++u) {
-            const int32_t item = base + u * nwarps;
-            live[u] = item < total_items;                       // warp-uniform
-            row[u] = live[u] ? item / chunks_per_row : 0;
-            col[u] = live[u] ? (item - row[u] * chunks_per_row) * 256 + lane * 8 : K;
-            v[u] = make_uint4(0u, 0u, 0u, 0u);
-            if (col[u] < K)
-                v[u] = __ldcs(reinterpret_cast<const uint4*>(x + static_cast<int64_t>(row[u]) * ld + col[u]));
+    for (int32_t unit = warp_global; unit < total_units; unit += nwarps) {
+        const int32_t row = unit >> split_log2;
+        const int32_t c_begin = (unit - (row << split_log2)) * chunks_per_unit;
+        const int32_t c_end = min(chunks_per_row, c_begin + chunks_per_unit);
+        if (c_begin >= c_end) continue;
+        float g = g_single, c1 = c1_single;
+        if (segs.nseg != 0) {
+            g = __ldg(g_ptr + seg_of(segs, row));
+            c1 = __fdiv_rn(1.0f, __fmul_rn(6.0f, g));
         }
+        const uint16_t* xrow = x + static_cast<int64_t>(row) * ld;
+        uint8_t* crow = codes + static_cast<int64_t>(row) * (K >> 1);
+        // scale bytes of this row: byte offset of block kb is sf_row + (kb >> 2) * 512 + (kb & 3)
+        // in the tensor-core layout, sf_row + kb in the linear one
+        uint8_t* sf_row = MMA_LAYOUT
+            ? sf + static_cast<int64_t>(row >> 7) * katoms * 512 + (row & 31) * 16 + ((row & 127) >> 5) * 4
+            : sf + static_cast<int64_t>(row) * KB;
+        for (int32_t c0 = c_begin; c0 < c_end; c0 += UNROLL) {
+            uint32_t v[UNROLL][8];
+            int32_t col[UNROLL];
 #pragma unroll
-        for (int u = 0; u < UNROLL; ++u) {
-            if (!live[u]) continue;                             // whole warp skips together
-            const float g = (segs.nseg == 0) ? g_single : __ldg(g_ptr + seg_of(segs, row[u]));
-            const float c1 = __fdiv_rn(1.0f, __fmul_rn(6.0f, g));
-            float f[8];
-            bf16x8_to_f32(v[u], f);
-            uint32_t s8;
-            const uint32_t word = quantize_slice(f, g, c1, s8);
-            const bool in_range = col[u] < K;
-            if (!in_range) s8 = 0u;
-            if (in_range)
-                *reinterpret_cast<uint32_t*>(codes + static_cast<int64_t>(row[u]) * (K >> 1) + (col[u] >> 1)) = word;
-            // scale bytes: the even lane of each pair holds the block's byte
-            const int l0 = lane & ~7;
-            const uint32_t w = __shfl_sync(0xffffffffu, s8, l0) | (__shfl_sync(0xffffffffu, s8, l0 + 2) << 8) |
-                               (__shfl_sync(0xffffffffu, s8, l0 + 4) << 16) |
-                               (__shfl_sync(0xffffffffu, s8, l0 + 6) << 24);
-            const int32_t kb = col[u] >> 4;
-            if (MMA_LAYOUT) {
-                if ((lane & 7) == 0 && kb < KB)                 // blocks past K inside the word are zero
-                    *reinterpret_cast<uint32_t*>(sf + sf_mma_offset(row[u], kb, katoms)) = w;
-            } else {
-                if ((lane & 1) == 0 && in_range) sf[static_cast<int64_t>(row[u]) * KB + kb] = static_cast<uint8_t>(s8);
+            for (int u = 0; u < UNROLL; ++u) {
+                col[u] = (c0 + u < c_end) ? (c0 + u) * 512 + lane * 16 : K;
+                if (col[u] < K) {
+                    ldg256_stream(xrow + col[u], v[u]);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) v[u][i] = 0u;
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                if (c0 + u >= c_end) break;                         // warp-uniform
+                uint32_t s8;
+                const uint2 word = quantize_block(v[u], g, c1, s8);
+                const bool in_range = col[u] < K;
+                if (!in_range) s8 = 0u;
+                if (in_range) *reinterpret_cast<uint2*>(crow + (col[u] >> 1)) = word;
+                const int32_t kb = col[u] >> 4;                     // this lane's block index
+                if (MMA_LAYOUT || ((KB & 3) == 0 && (reinterpret_cast<uintptr_t>(sf) & 3u) == 0)) {
+                    // four neighbouring lanes hold the four scale bytes of one 32-bit word
+                    uint32_t w = s8 | (__shfl_down_sync(0xffffffffu, s8, 1) << 8);
+                    w |= __shfl_down_sync(0xffffffffu, w, 2) << 16;
+                    if ((lane & 3) == 0 && kb < KB) {
+                        if (MMA_LAYOUT) *reinterpret_cast<uint32_t*>(sf_row + static_cast<int64_t>(kb >> 2) * 512) = w;
+                        else            *reinterpret_cast<uint32_t*>(sf_row + kb) = w;
+                    }
+                } else if (in_range) {
+                    sf_row[kb] = static_cast<uint8_t>(s8);
+                }
             }
         }
     }

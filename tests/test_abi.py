@@ -54,8 +54,8 @@ def test_host_side_argument_checks_need_no_gpu(L):
     assert L.nvfp4_calibrate(p, 4, 16, 8, p, None, None) == 2                      # ld < cols
     assert L.nvfp4_quantize_act(p, 4, 24, 24, p, p, p, nv.SF_MMA, None) == 2      # K % 16
     assert L.nvfp4_quantize_act(None, 4, 32, 32, p, p, p, nv.SF_MMA, None) == 1
-    assert L.nvfp4_quantize_act(p, 4, 32, 36, p, p, p, nv.SF_MMA, None) == 3      # ld % 8
-    assert L.nvfp4_quantize_act(vp(0x1008), 4, 32, 32, p, p, p, nv.SF_MMA, None) == 3
+    assert L.nvfp4_quantize_act(p, 4, 32, 40, p, p, p, nv.SF_MMA, None) == 3      # ld % 16
+    assert L.nvfp4_quantize_act(vp(0x1010), 4, 32, 32, p, p, p, nv.SF_MMA, None) == 3   # 16- but not 32-byte aligned
     assert L.nvfp4_quantize_act(p, 4, 32, 32, p, p, p, 7, None) == 9
     assert L.nvfp4_quantize_weight(p, 16, 32, 32, seg, 2, p, 0, p, p, nv.SF_MMA, None) != 4
     seg[1].col_begin = 9

@@ -50,7 +50,7 @@ def test_ragged_shapes(M, K, layout):
 
 def test_strided_input():
     x = synth.prefill_activations(1, 3, 70, 320)
-    _act_case(x, ld_pad=24)
+    _act_case(x, ld_pad=48)
 
 
 def test_every_finite_bf16_pattern_at_several_scales():
