@@ -259,28 +259,39 @@ nvfp4_status quantize_impl(const void* d_x, int64_t M, int64_t K, int64_t ld, co
             cudaSuccess)
             return NVFP4_ERR_CUDA;
     }
-    // a unit = up to `per_unit` consecutive chunks of one row; units per row rounded up to a power of two
+    // a unit = up to `per_unit` consecutive chunks of one row, handled by one warp
     constexpr int kUnroll = 2;
-    const int64_t resident_warps = static_cast<int64_t>(info.sm_count) * 48;
-    int64_t per_unit = (M * chunks > 2 * resident_warps) ? kUnroll : 1;
-    int split_log2 = 0;
-    while ((1ll << split_log2) * per_unit < chunks) ++split_log2;
-    per_unit = (chunks + (1ll << split_log2) - 1) >> split_log2;
-    const int64_t units = M << split_log2;
+    const int64_t resident_warps = static_cast<int64_t>(info.sm_count) * 40;   // 5 blocks of 8 warps per SM
+    const int64_t per_unit = (M * chunks > 2 * resident_warps) ? kUnroll : 1;
+    const int64_t units_per_row = (chunks + per_unit - 1) / per_unit;
+    const int64_t units = M * units_per_row;
     if (units >= (1ll << 31)) return NVFP4_ERR_SHAPE;
     int64_t blocks = (units + 7) / 8;
-    const int64_t max_blocks = static_cast<int64_t>(info.sm_count) * 6;
+    // persistent grid: exactly what is resident at once, so that no partial second wave forms
+    static std::atomic<int> per_sm_mma{0}, per_sm_lin{0};
+    std::atomic<int>& per_sm_slot = (layout == NVFP4_SF_MMA) ? per_sm_mma : per_sm_lin;
+    int per_sm = per_sm_slot.load(std::memory_order_relaxed);
+    if (per_sm == 0) {
+        cudaError_t e = (layout == NVFP4_SF_MMA)
+            ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, quantize_kernel<true, kUnroll>, 256, 0)
+            : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, quantize_kernel<false, kUnroll>, 256, 0);
+        if (e != cudaSuccess || per_sm < 1) { cudaGetLastError(); per_sm = 4; }
+        per_sm_slot.store(per_sm, std::memory_order_relaxed);
+    }
+    const int64_t max_blocks = static_cast<int64_t>(info.sm_count) * per_sm;
     if (blocks > max_blocks) blocks = max_blocks;
     if (blocks < 1) blocks = 1;
     const uint16_t* x = reinterpret_cast<const uint16_t*>(d_x);
     if (layout == NVFP4_SF_MMA)
         quantize_kernel<true, kUnroll><<<static_cast<int>(blocks), 256, 0, stream>>>(
             x, static_cast<int32_t>(M), static_cast<int32_t>(K), ld, d_g, segs, d_codes, d_sf,
-            static_cast<int32_t>(chunks), static_cast<int32_t>(per_unit), split_log2, static_cast<int32_t>(units));
+            static_cast<int32_t>(chunks), static_cast<int32_t>(per_unit), static_cast<int32_t>(units_per_row),
+            static_cast<int32_t>(units));
     else
         quantize_kernel<false, kUnroll><<<static_cast<int>(blocks), 256, 0, stream>>>(
             x, static_cast<int32_t>(M), static_cast<int32_t>(K), ld, d_g, segs, d_codes, d_sf,
-            static_cast<int32_t>(chunks), static_cast<int32_t>(per_unit), split_log2, static_cast<int32_t>(units));
+            static_cast<int32_t>(chunks), static_cast<int32_t>(per_unit), static_cast<int32_t>(units_per_row),
+            static_cast<int32_t>(units));
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }

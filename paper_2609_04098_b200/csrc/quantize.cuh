@@ -117,13 +117,13 @@ __device__ __forceinline__ uint2 quantize_block(const uint32_t (&v)[8], float g,
 }
 
 // A warp owns `chunks_per_unit` consecutive 512-element chunks of one row (a "unit"); units are
-// dealt round-robin to a persistent grid.  split_log2: log2 of the units per row.
+// dealt round-robin to a persistent grid.
 template <bool MMA_LAYOUT, int UNROLL>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 5)
 quantize_kernel(const uint16_t* __restrict__ x, int32_t M, int32_t K, int64_t ld,
                 const float* __restrict__ g_ptr, SegTable segs,
                 uint8_t* __restrict__ codes, uint8_t* __restrict__ sf,
-                int32_t chunks_per_row, int32_t chunks_per_unit, int32_t split_log2, int32_t total_units) {
+                int32_t chunks_per_row, int32_t chunks_per_unit, int32_t units_per_row, int32_t total_units) {
     const int lane = threadIdx.x & 31;
     const int32_t warp_global = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int32_t nwarps = gridDim.x * (blockDim.x >> 5);
@@ -133,10 +133,9 @@ quantize_kernel(const uint16_t* __restrict__ x, int32_t M, int32_t K, int64_t ld
     const float c1_single = __fdiv_rn(1.0f, __fmul_rn(6.0f, g_single));
 
     for (int32_t unit = warp_global; unit < total_units; unit += nwarps) {
-        const int32_t row = unit >> split_log2;
-        const int32_t c_begin = (unit - (row << split_log2)) * chunks_per_unit;
+        const int32_t row = unit / units_per_row;                  // one division per >= 512 elements
+        const int32_t c_begin = (unit - row * units_per_row) * chunks_per_unit;
         const int32_t c_end = min(chunks_per_row, c_begin + chunks_per_unit);
-        if (c_begin >= c_end) continue;
         float g = g_single, c1 = c1_single;
         if (segs.nseg != 0) {
             g = __ldg(g_ptr + seg_of(segs, row));
