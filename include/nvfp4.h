@@ -161,6 +161,39 @@ nvfp4_status nvfp4_linear_bf16(const void* d_x, int64_t ldx, const float* d_g_a,
 size_t nvfp4_linear_bf16_workspace_bytes(int64_t M, int64_t N, int64_t K, int nseg);
 
 /*
+ * nvfp4_linear_bf16 for callers that cannot provide a workspace.  (The paper has no
+ * counterpart for this call; it exists for integration only.)
+ *
+ * Some hosts of this library may not allocate device memory at the point where they
+ * run a layer: an inference server that has handed all device memory to its own pool,
+ * a plug-in running inside another framework's execution callback, code between
+ * allocator-frozen phases of a serving loop.  They have nowhere to get the scratch
+ * buffer that nvfp4_linear_bf16 needs for the quantized activations.  This variant
+ * takes the same inputs and outputs and keeps that scratch in a fixed array inside
+ * the library's own device image, NVFP4_STATIC_SCRATCH_BYTES large; every GPU that
+ * loads the library holds the array until the process exits.
+ *
+ *   - It calls no cudaMalloc / cudaFree and no allocating library routine.
+ *   - Sizes whose nvfp4_linear_bf16_workspace_bytes(M, N, K, nseg) exceeds
+ *     NVFP4_STATIC_SCRATCH_BYTES are rejected with NVFP4_ERR_WORKSPACE before anything
+ *     is launched (the limit fits decode-sized batches, e.g. M = 256 rows at K = 16384).
+ *   - The first call on each device looks up the array's device address (once, with that
+ *     device current).  Make that first call outside of any stream capture.
+ *   - All calls share the one array and it keeps the previous call's contents; the
+ *     status word at its start is cleared by every call.  Two calls that overlap on the
+ *     GPU (different streams, no dependency) race on it: serialise them.
+ *   - nvfp4_static_status(stream) is nvfp4_device_status for this array.
+ * Everything else (arguments, layouts, errors) is as for nvfp4_linear_bf16.
+ */
+#define NVFP4_STATIC_SCRATCH_BYTES (4u * 1024u * 1024u)
+nvfp4_status nvfp4_linear_bf16_static(const void* d_x, int64_t ldx, const float* d_g_a,
+                                      int64_t M, int64_t K,
+                                      const uint8_t* d_w_codes, const uint8_t* d_w_sf, int64_t N,
+                                      const nvfp4_segment* segs, const float* d_g_seg, int nseg,
+                                      void* d_y, int64_t ldy, uint32_t flags, void* stream);
+nvfp4_status nvfp4_static_status(void* stream);
+
+/*
  * Clears the status word of a workspace (enqueue before the first nvfp4_linear* that
  * uses it; the kernels only ever set it).
  */

@@ -25,7 +25,7 @@ MAX_SEGMENTS = 32
 EXPORTS = (
     "nvfp4_sf_bytes", "nvfp4_calibrate", "nvfp4_quantize_act", "nvfp4_quantize_weight",
     "nvfp4_linear", "nvfp4_linear_workspace_bytes", "nvfp4_linear_bf16",
-    "nvfp4_linear_bf16_workspace_bytes", "nvfp4_workspace_reset", "nvfp4_device_status",
+    "nvfp4_linear_bf16_workspace_bytes", "nvfp4_linear_bf16_static", "nvfp4_static_status", "nvfp4_workspace_reset", "nvfp4_device_status",
     "nvfp4_launch_count", "nvfp4_set_gemm_variant", "nvfp4_gemm_variants", "nvfp4_status_string",
 )
 
@@ -69,6 +69,10 @@ def lib() -> ctypes.CDLL:
     L.nvfp4_linear_bf16.argtypes = [vp, i64, vp, i64, i64, vp, vp, i64, segp, vp, i32, vp, i64, u32, vp, sz, vp]
     L.nvfp4_linear_bf16_workspace_bytes.restype = sz
     L.nvfp4_linear_bf16_workspace_bytes.argtypes = [i64, i64, i64, i32]
+    L.nvfp4_linear_bf16_static.restype = i32
+    L.nvfp4_linear_bf16_static.argtypes = [vp, i64, vp, i64, i64, vp, vp, i64, segp, vp, i32, vp, i64, u32, vp]
+    L.nvfp4_static_status.restype = i32
+    L.nvfp4_static_status.argtypes = [vp]
     L.nvfp4_workspace_reset.restype = i32
     L.nvfp4_workspace_reset.argtypes = [vp, sz, vp]
     L.nvfp4_device_status.restype = i32
@@ -208,6 +212,36 @@ def nvfp4_linear_bf16(x, g_a, w_codes, w_sf, segments, g_seg, workspace, out=Non
                                    _segments(pairs), _ptr(g_seg), len(pairs), _ptr(out), out.stride(0), flags,
                                    _ptr(workspace), workspace.numel(), _stream(stream)), "nvfp4_linear_bf16")
     return out
+
+
+STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
+
+
+def nvfp4_linear_bf16_static(x, g_a, w_codes, w_sf, segments, g_seg, out=None, out_f32: bool = False,
+                             stream=None) -> torch.Tensor:
+    """``nvfp4_linear_bf16`` without a caller-provided workspace, for hosts that may not allocate
+    device memory when they run a layer (a server whose memory pool owns the whole device, a
+    plug-in inside another framework's callback).  The quantized activations go to a fixed
+    ``STATIC_SCRATCH_BYTES`` array inside the library; larger problems raise ``Nvfp4Error``
+    (workspace).  Calls share that array, so calls that overlap on the GPU must be serialised;
+    make the first call on a device outside of stream capture.  ``out`` must be passed in by a
+    caller that really cannot allocate (otherwise it is allocated here, by torch)."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
+    M, K = x.shape
+    N = w_codes.shape[0]
+    pairs = seg_pairs(segments)
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.float32 if out_f32 else torch.bfloat16, device=x.device)
+    flags = OUT_F32 if out.dtype == torch.float32 else OUT_BF16
+    _check(lib().nvfp4_linear_bf16_static(_ptr(x), x.stride(0), _ptr(g_a), M, K, _ptr(w_codes), _ptr(w_sf), N,
+                                          _segments(pairs), _ptr(g_seg), len(pairs), _ptr(out), out.stride(0),
+                                          flags, _stream(stream)), "nvfp4_linear_bf16_static")
+    return out
+
+
+def static_status(stream=None) -> int:
+    """Status word of the library's static scratch (synchronises the stream)."""
+    return int(lib().nvfp4_static_status(_stream(stream)))
 
 
 def workspace_reset(workspace: torch.Tensor, stream=None) -> None:

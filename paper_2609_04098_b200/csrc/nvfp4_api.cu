@@ -496,6 +496,54 @@ nvfp4_status nvfp4_linear_bf16(const void* d_x, int64_t ldx, const float* d_g_a,
                         d_workspace, kStatusBytes, stream);
 }
 
+// ---------------------------------------------------------------- no-allocation variant
+// Scratch for nvfp4_linear_bf16_static.  In host code this name is only a stand-in for the
+// symbol: the device address comes from cudaGetSymbolAddress, per device.
+static __device__ __align__(256) unsigned char g_static_scratch[NVFP4_STATIC_SCRATCH_BYTES];
+
+namespace {
+nvfp4_status static_scratch_address(void** out) {
+    static std::mutex mu;
+    static std::unordered_map<int, void*> by_device;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return NVFP4_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    auto it = by_device.find(dev);
+    if (it != by_device.end()) { *out = it->second; return NVFP4_OK; }
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || ptr == nullptr) {
+        cudaGetLastError();
+        return NVFP4_ERR_CUDA;
+    }
+    by_device[dev] = ptr;
+    *out = ptr;
+    return NVFP4_OK;
+}
+}  // namespace
+
+nvfp4_status nvfp4_linear_bf16_static(const void* d_x, int64_t ldx, const float* d_g_a, int64_t M, int64_t K,
+                                      const uint8_t* d_w_codes, const uint8_t* d_w_sf, int64_t N,
+                                      const nvfp4_segment* segs, const float* d_g_seg, int nseg, void* d_y,
+                                      int64_t ldy, uint32_t flags, void* stream) {
+    if (M < 0 || K <= 0 || (K % 64) != 0) return NVFP4_ERR_SHAPE;
+    const size_t need = nvfp4_linear_bf16_workspace_bytes(M, N, K, nseg);
+    if (need == 0 || need > NVFP4_STATIC_SCRATCH_BYTES) return NVFP4_ERR_WORKSPACE;   // beyond the fixed array
+    void* scratch = nullptr;
+    nvfp4_status st = static_scratch_address(&scratch);
+    if (st != NVFP4_OK) return st;
+    st = nvfp4_workspace_reset(scratch, NVFP4_STATIC_SCRATCH_BYTES, stream);           // status word starts at zero
+    if (st != NVFP4_OK) return st;
+    return nvfp4_linear_bf16(d_x, ldx, d_g_a, M, K, d_w_codes, d_w_sf, N, segs, d_g_seg, nseg, d_y, ldy, flags,
+                             scratch, NVFP4_STATIC_SCRATCH_BYTES, stream);
+}
+
+nvfp4_status nvfp4_static_status(void* stream) {
+    void* scratch = nullptr;
+    nvfp4_status st = static_scratch_address(&scratch);
+    if (st != NVFP4_OK) return st;
+    return nvfp4_device_status(scratch, stream);
+}
+
 nvfp4_status nvfp4_device_status(const void* d_workspace, void* stream) {
     if (d_workspace == nullptr) return NVFP4_ERR_NULL;
     uint32_t word = 0;
