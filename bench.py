@@ -204,6 +204,7 @@ def run_gpu(args):
     if args.workload == "mlp":
         wl = MlpPair(args.tokens)
         host = wl.host_inputs(args.seed)
+        cpu_x, cpu_w = host["x1"], host["w_gu"]
         x1, x2 = up(host["x1"]), up(host["x2"])
         w_gu_c, w_gu_sf, g_gu = nv.nvfp4_quantize_weight(up(host["w_gu"]), wl.seg_gu)
         w_d_c, w_d_sf, g_d = nv.nvfp4_quantize_weight(up(host["w_d"]), wl.seg_d)
@@ -240,6 +241,7 @@ def run_gpu(args):
         wl = GdnProj(args.tokens) if args.workload == "gdn" else OneLinear(args.tokens)
         hx = synth.prefill_activations(args.seed, 401, wl.M, HIDDEN)
         hw = synth.weights(args.seed, 402, wl.segs, HIDDEN)
+        cpu_x, cpu_w = hx, hw
         # rotate through enough distinct activation/output sets to exceed L2
         per_set = wl.M * HIDDEN * 2 + wl.M * wl.N * 2
         nset = max(1, min(8, int(np.ceil(300e6 / per_set))))
@@ -407,7 +409,8 @@ def run_gpu(args):
 
     if rank == 0:
         if not args.skip_cpu:
-            result["cpu_baseline"] = cpu_baseline(wl, target_s=args.cpu_seconds, seed=args.seed)
+            result["cpu_baseline"] = cpu_baseline(wl, target_s=args.cpu_seconds, seed=args.seed,
+                                                  x_bits=cpu_x, w_bits=cpu_w)
         line = {"metric": "nvfp4_w4a4_linear_tflops", "value": round(value, 2), "unit": "TFLOP/s",
                 "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
                 "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak",
@@ -425,37 +428,40 @@ def run_gpu(args):
 
 
 # --------------------------------------------------------------------------- CPU oracle arm
-def cpu_baseline(wl, target_s=15.0, seed=0):
-    """The oracle as it stands, timed on a bounded sample of the same workload:
-    quantize R activation rows, then the exact GEMM of those rows against a slice of
-    the first layer's weight rows."""
+def cpu_baseline(wl, target_s=15.0, seed=0, x_bits=None, w_bits=None):
+    """The oracle as it stands, timed on a bounded sample of the same workload: quantize R
+    activation rows of the first layer's input and run the exact GEMM of those rows against
+    ALL of that layer's (oracle-quantized) weight rows.  R is sized for about `target_s`
+    seconds from a small trial.  Weight quantization is setup (offline in the path), untimed."""
     import oracle
     K = HIDDEN
     segs = wl.seg_gu if hasattr(wl, "seg_gu") else wl.segs
-    n_full = sum(s.count for s in segs)
-    ncols = min(n_full, 2048)
-    w = synth.weights(seed, 302, synth.make_segments((("w", ncols, 0.02),)), K)
-    _, gw = oracle.calibrate(w)
-    wc, wsf = oracle.quantize(w, oracle.row_scales(ncols, g=gw))
-    gcol = np.full(ncols, gw, np.float32)
+    N = sum(s.count for s in segs)
+    if w_bits is None:
+        w_bits = synth.weights(seed, 302 if hasattr(wl, "seg_gu") else 402, segs, K)
+    if x_bits is None:
+        x_bits = synth.prefill_activations(seed, 301 if hasattr(wl, "seg_gu") else 401, min(wl.M, 8192), K)
+    gs = [oracle.calibrate(w_bits[s.begin:s.begin + s.count])[1] for s in segs]
+    wc, wsf = oracle.quantize(w_bits, oracle.row_scales(N, segs, gs))
+    gcol = oracle.col_scales(N, segs, gs)
 
     def run(rows):
-        x = synth.prefill_activations(seed, 301, rows, K)
+        x = x_bits[:rows]
         t0 = time.perf_counter()
         _, ga = oracle.calibrate(x)
         ac, asf = oracle.quantize(x, oracle.row_scales(rows, g=ga))
         oracle.gemm(ac, asf, ga, wc, wsf, gcol)
         return time.perf_counter() - t0
 
-    t_small = run(8)
-    t_small = min(t_small, run(8))
-    rows = int(max(8, min(65536, 8 * target_s / max(t_small, 1e-4))))
-    t = run(rows)
-    flops = gemm_flops(rows, ncols, K)
+    trial = min(32, x_bits.shape[0])
+    t_trial = run(trial)
+    rows = int(max(trial, min(x_bits.shape[0], trial * target_s / max(t_trial, 1e-3))))
+    t = run(rows) if rows > trial else t_trial
+    flops = gemm_flops(rows, N, K)
     return {"value": round(flops / t / 1e12, 6), "unit": "TFLOP/s", "cores": oracle.num_threads(),
             "kind": "oracle", "seconds": round(t, 2),
-            "sample": "quantize + exact GEMM of %d token rows x %d weight rows (K=%d) of the first layer" % (
-                rows, ncols, K)}
+            "sample": "quantize + exact GEMM of %d token rows x all %d weight rows (K=%d) of the step's first layer" % (
+                rows, N, K)}
 
 
 def run_reference(args):
@@ -464,12 +470,16 @@ def run_reference(args):
     if int(os.environ.get("RANK", "0")) != 0:
         return
     wl = {"mlp": MlpPair, "gdn": GdnProj, "linear": OneLinear}[args.workload](args.tokens)
-    per_step_s = max(2.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    per_step_s = max(1.0, min(15.0, 100.0 / max(1, args.steps + args.warmup)))
+    segs = wl.seg_gu if hasattr(wl, "seg_gu") else wl.segs
+    mlp = hasattr(wl, "seg_gu")
+    w_bits = synth.weights(args.seed, 302 if mlp else 402, segs, HIDDEN)
+    x_bits = synth.prefill_activations(args.seed, 301 if mlp else 401, min(wl.M, 8192), HIDDEN)
     for _ in range(args.warmup):
-        cpu_baseline(wl, target_s=per_step_s / 4, seed=args.seed)
+        cpu_baseline(wl, target_s=per_step_s / 4, seed=args.seed, x_bits=x_bits, w_bits=w_bits)
     vals, secs, last = [], [], None
     for _ in range(args.steps):
-        last = cpu_baseline(wl, target_s=per_step_s, seed=args.seed)
+        last = cpu_baseline(wl, target_s=per_step_s, seed=args.seed, x_bits=x_bits, w_bits=w_bits)
         vals.append(last["value"])
         secs.append(last["seconds"])
     value = float(np.mean(vals))
@@ -487,8 +497,8 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="mlp", choices=["mlp", "gdn", "linear"])
     ap.add_argument("--tokens", type=int, default=8192)
@@ -498,6 +508,11 @@ def main():
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--skip-quantize", action="store_true")
     args = ap.parse_args()
+    ref = args.impl == "reference"
+    if args.steps is None:
+        args.steps = 3 if ref else 200
+    if args.warmup is None:
+        args.warmup = 1 if ref else 10
     if args.impl == "reference":
         run_reference(args)
     else:
