@@ -30,6 +30,7 @@
 // tells its partner instead of hanging.
 #pragma once
 #include <cstdint>
+#include <type_traits>
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -50,6 +51,7 @@ struct GemmParams {
     int32_t n_tiles;         // ceil(N / BN)
     int32_t k_tiles;         // ceil(K / 256)
     int32_t katoms;          // K / 64: 512-byte scale atoms per 128-row band
+    int32_t group_m;         // row units per raster group (see tile_of)
     uint32_t flags;
     uint32_t tma_store;      // 1: bf16 output through the TMA-store path (tmY valid)
     int32_t nseg;
@@ -83,7 +85,14 @@ constexpr int kOutPieceBytes = 32 * kOutPieceCols * 2;
 
 template <int BN, int STAGES, bool PAIR>
 struct GemmCfg {
-    static constexpr int ACC = (BN == 128) ? 2 : 1;                    // TMEM accumulators
+    // Two TMEM accumulators.  BN = 128: disjoint (0..127, 128..255).  BN = 256: they do not both
+    // fit beside the scale columns, so they OVERLAP by one epilogue piece: columns 0..255 and
+    // 192..447.  The epilogue drains the shared 64 columns of a tile first and only then lets
+    // the next tile's MMAs start; the rest of its drain runs under those MMAs.
+    static constexpr int ACC = 2;
+    static constexpr bool OVERLAP = (BN == 256);
+    static constexpr int ACC_STRIDE = OVERLAP ? BN - kOutPieceCols : BN;
+    static constexpr int SF_SETS = OVERLAP ? 1 : STAGES;               // sets of scale columns
     static constexpr int B_ROWS = PAIR ? BN / 2 : BN;                  // W rows this CTA loads
     static constexpr int NB_BANDS = BN / 128;                          // 128-row scale bands of the W tile
     static constexpr int CTAS = PAIR ? 2 : 1;
@@ -95,14 +104,16 @@ struct GemmCfg {
     static constexpr int OUT_BYTES = 4 * 2 * kOutPieceBytes;           // per epilogue warp: two pieces
     static constexpr int BAR_BYTES = (2 * STAGES + 2 * ACC + 1) * 8 + 16;
     static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + OUT_BYTES + BAR_BYTES;
-    // TMEM columns: accumulators first, then one set of scale columns per smem stage
+    // TMEM columns: accumulators first, then the scale columns (one set per smem stage, or a
+    // single set that every stage reuses: the copies into it are ordered behind the MMAs that
+    // read it because both are issued by one thread into the same pipe)
     static constexpr int SFA_SET_COLS = kStepsPerStage * 4;
     static constexpr int SFB_SET_COLS = kStepsPerStage * (BN / 32);
-    static constexpr int SFA_COL0 = ACC * BN;
-    static constexpr int SFB_COL0 = SFA_COL0 + STAGES * SFA_SET_COLS;
+    static constexpr int SFA_COL0 = ACC_STRIDE + BN;
+    static constexpr int SFB_COL0 = SFA_COL0 + SF_SETS * SFA_SET_COLS;
     static_assert(BN == 128 || BN == 256, "BN must be 128 or 256");
     static_assert(!PAIR || BN == 256, "the pair kernel uses 256 x 256 tiles");
-    static_assert(SFB_COL0 + STAGES * SFB_SET_COLS <= kTmemCols, "TMEM budget");
+    static_assert(SFB_COL0 + SF_SETS * SFB_SET_COLS <= kTmemCols, "TMEM budget");
     static_assert(SMEM_BYTES <= 232448, "shared memory budget");
     static_assert(STAGE_BYTES % 1024 == 0, "stage alignment");
 };
@@ -166,12 +177,19 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    // tile index -> (row unit, column tile); row units vary fastest so that the CTAs running
-    // at the same time share W tiles through L2
+    // tile index -> (row unit, column tile).  Tiles are visited in groups of `group_m` row
+    // units; inside a group the row unit varies fastest, then the column tile.  The CTAs that
+    // run at the same time then share W tiles through L2, and the A rows of one group (sized
+    // by the host to a fraction of L2) stay resident while the group sweeps all of W.
+    const uint32_t group_m = static_cast<uint32_t>(p.group_m);
+    const uint32_t tiles_per_group = group_m * static_cast<uint32_t>(p.n_tiles);
     auto tile_of = [&](uint32_t t, int32_t& um, int32_t& un) {
         const uint32_t tile = unit_id + t * n_units;
-        um = static_cast<int32_t>(tile % m_units);
-        un = static_cast<int32_t>(tile / m_units);
+        const uint32_t group = tile / tiles_per_group, r = tile - group * tiles_per_group;
+        const uint32_t first = group * group_m;
+        const uint32_t gsize = min(group_m, m_units - first);
+        un = static_cast<int32_t>(r / gsize);
+        um = static_cast<int32_t>(first + (r - static_cast<uint32_t>(un) * gsize));
     };
 
     if (warp == 4 || warp == 5) {
@@ -247,14 +265,20 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             auto desc = [](uint32_t lo, uint32_t hi) { return (static_cast<uint64_t>(hi) << 32) | lo; };
             const int32_t tail_steps = p.katoms - (p.k_tiles - 1) * kStepsPerStage;   // K-steps of a tile's last stage
             bool ok = true;
-            uint32_t it = 0, kt = 0, acc = 0, aph = 0, ph = 0;
+            uint32_t it = 0, kt = 0, tl = 0, ph = 0;
             bool have_full = false;          // the coming iteration's "stage full" was already observed
             while (ok && it < total_it) {
 #pragma unroll
                 for (int s = 0; s < STAGES; ++s) {
                     if (it >= total_it) break;
+                    const uint32_t acc = tl & 1u;
                     if (kt == 0) {
-                        if (!ptx::mbar_wait_bounded(&tempty[acc], aph ^ 1u, abort_flag, p.wait_limit_ns, peer_abort)) { ok = false; break; }
+                        // disjoint accumulators: wait until tile tl-2 (same accumulator) is drained;
+                        // overlapping ones: until tile tl-1 has given up the shared columns
+                        const uint32_t dep = C::OVERLAP ? tl - 1u : tl - 2u;
+                        if (tl >= (C::OVERLAP ? 1u : 2u)) {
+                            if (!ptx::mbar_wait_bounded(&tempty[dep & 1u], (dep >> 1) & 1u, abort_flag, p.wait_limit_ns, peer_abort)) { ok = false; break; }
+                        }
                         if (have_full) ptx::tc_fence_after();
                     }
                     if (!have_full) {
@@ -264,9 +288,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     have_full = false;
                     if (leader) NVFP4_TRACE(p, 2, it);
                     const uint32_t st_enc = smem_enc + s * (C::STAGE_BYTES >> 4);
-                    const uint32_t sfa_t = tmem_base + C::SFA_COL0 + s * C::SFA_SET_COLS;
-                    const uint32_t sfb_t = tmem_base + C::SFB_COL0 + s * C::SFB_SET_COLS;
-                    const uint32_t d_tmem = tmem_base + acc * BN;
+                    const uint32_t sfa_t = tmem_base + C::SFA_COL0 + (C::SF_SETS == 1 ? 0 : s) * C::SFA_SET_COLS;
+                    const uint32_t sfb_t = tmem_base + C::SFB_COL0 + (C::SF_SETS == 1 ? 0 : s) * C::SFB_SET_COLS;
+                    const uint32_t d_tmem = tmem_base + acc * C::ACC_STRIDE;
                     const bool last_kt = kt + 1 == k_tiles;
                     const int32_t steps = last_kt ? tail_steps : kStepsPerStage;
 #pragma unroll
@@ -317,12 +341,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                         NVFP4_TRACE(p, 3, it);
                     }
                     ++it;
-                    if (last_kt) {
-                        kt = 0;
-                        if (ACC == 1) { aph ^= 1u; } else { acc ^= 1u; if (acc == 0u) aph ^= 1u; }
-                    } else {
-                        ++kt;
-                    }
+                    if (last_kt) { kt = 0; ++tl; } else { ++kt; }
                 }
                 ph ^= 1u;
             }
@@ -346,7 +365,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             int32_t um, un;
             tile_of(t, um, un);
             const int32_t n0 = un * BN;
-            const uint32_t acc = t % ACC, aph = (t / ACC) & 1u;
+            const uint32_t acc = t & 1u, aph = (t >> 1) & 1u;
             if (warp == 0 && lane == 0) NVFP4_TRACE(p, 7, t);
             // global scale of columns n0 + 32 i + lane, i = 0 .. BN/32-1, in registers
             float areg[BN / 32];
@@ -369,20 +388,25 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             if (!ok) break;
             ptx::tc_fence_after();
             if (warp == 0 && lane == 0) NVFP4_TRACE(p, 6, t);
-            const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * BN;
+            const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * C::ACC_STRIDE;
             const int32_t row0 = (PAIR ? 2 * um + static_cast<int32_t>(rank) : um) * kBM + quarter * 32;
             constexpr int NP = BN / kOutPieceCols;
+            // piece order: with overlapping accumulators the shared columns go first (the last piece
+            // of the lower accumulator, the first piece of the upper one)
+            auto drain = [&](auto first_c) {
+            constexpr int first_piece = decltype(first_c)::value;
             uint32_t ra[64], rb[64];
-            ptx::tmem_ld_32x64(t_row, ra);
+            ptx::tmem_ld_32x64(t_row + first_piece * kOutPieceCols, ra);
 #pragma unroll
-            for (int pc = 0; pc < NP; ++pc) {
-                uint32_t (&cur)[64] = (pc & 1) ? rb : ra;
-                uint32_t (&nxt)[64] = (pc & 1) ? ra : rb;
+            for (int k = 0; k < NP; ++k) {
+                uint32_t (&cur)[64] = (k & 1) ? rb : ra;
+                uint32_t (&nxt)[64] = (k & 1) ? ra : rb;
+                const int pc = (first_piece + k) % NP;               // this piece; next is (pc + 1) % NP
                 ptx::tmem_ld_wait();
-                if (pc + 1 < NP) {
-                    ptx::tmem_ld_32x64(t_row + (pc + 1) * kOutPieceCols, nxt);
-                } else {
-                    // last column is in registers: hand the accumulator back to the MMA issuer
+                if (k + 1 < NP) ptx::tmem_ld_32x64(t_row + ((pc + 1) % NP) * kOutPieceCols, nxt);
+                if (C::OVERLAP ? (k == 0) : (k + 1 == NP)) {
+                    // overlapping: the shared columns are in registers, the next tile's MMAs may start;
+                    // disjoint: the whole accumulator is in registers
                     ptx::tc_fence_before();
                     __syncwarp();
                     if (lane == 0) {
@@ -432,6 +456,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     }
                 }
             }
+            };
+            if (C::OVERLAP && acc == 0u) drain(std::integral_constant<int, NP - 1>{});
+            else                         drain(std::integral_constant<int, 0>{});
         }
         if (use_tma && lane == 0) ptx::bulk_wait_group<0>();   // all output stores complete before exit
     }

@@ -199,6 +199,14 @@ nvfp4_status launch_gemm(const GemmMaps& tm, GemmParams& p, int sm_count, cudaSt
     p.n_tiles = (p.N + BN - 1) / BN;
     const int64_t m_units = PAIR ? (p.m_tiles + 1) / 2 : p.m_tiles;
     const int64_t tiles = m_units * p.n_tiles;
+    {
+        // rows of A kept live per raster group: about 32 MB of codes and scales (a quarter of L2)
+        const int64_t unit_bytes = static_cast<int64_t>(PAIR ? 256 : 128) * (p.K / 2 + p.K / 16);
+        int64_t g = (32ll << 20) / (unit_bytes > 0 ? unit_bytes : 1);
+        if (g < 1) g = 1;
+        if (g > m_units) g = m_units;
+        p.group_m = static_cast<int32_t>(g);
+    }
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof(cfg));
     cudaLaunchAttribute attr[1];
