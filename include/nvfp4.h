@@ -104,6 +104,24 @@ nvfp4_status nvfp4_quantize_act(const void* d_x, int64_t M, int64_t K, int64_t l
                                 nvfp4_sf_layout layout, void* stream);
 
 /*
+ * Activation quantization fused into its producer (paper: Background -- the MLP is among the
+ * 496 quantized linears, so the down projection's input silu(gate)*up is quantized on every
+ * call; Section 9 names activation quantization as the overhead to remove).  Reads the fused
+ * gate/up GEMM output once and writes only codes and scales: h is never stored in bf16.
+ *     h = bf16_rne( silu(gate) * up ),  then exactly nvfp4_quantize_act(h)
+ * with silu(g)*u evaluated in binary32 as: t = clamp(-g, -87, 87); n = rint(t*log2e);
+ * r = fmaf(t, log2e, -n); e = poly5(r) * 2^n; s = g * (1/(1+e)); s*u   (every step one IEEE op).
+ *   d_gate_up  bf16 [M, 2*inner], gate in columns [0, inner), up in [inner, 2*inner); row
+ *              stride ld >= 2*inner; 32-byte aligned, ld % 16 == 0, inner % 16 == 0
+ *   d_g        in: global scale of h (calibrated offline, as for any activation)
+ *   d_codes    out [M, inner/2]; d_sf out nvfp4_sf_bytes(M, inner, layout)
+ * Errors: as nvfp4_quantize_act.
+ */
+nvfp4_status nvfp4_swiglu_quantize(const void* d_gate_up, int64_t M, int64_t inner, int64_t ld,
+                                   const float* d_g, uint8_t* d_codes, uint8_t* d_sf,
+                                   nvfp4_sf_layout layout, void* stream);
+
+/*
  * Offline weight quantization, same format, blocks along K, with one global scale
  * per fused module (paper: Section 6 -- the calibration tool keeps one FP32 global
  * scale per linear module; the modules are later served as one fused GEMM).

@@ -62,6 +62,10 @@ def _load():
     L.orc_calibrate.argtypes = [u16p, i64, i64, i64, f32p, f32p]
     L.orc_quantize.restype = ctypes.c_int
     L.orc_quantize.argtypes = [u16p, i64, i64, i64, f32p, u8p, u8p]
+    L.orc_silu_mul.restype = ctypes.c_float
+    L.orc_silu_mul.argtypes = [ctypes.c_float, ctypes.c_float]
+    L.orc_swiglu_bf16.restype = None
+    L.orc_swiglu_bf16.argtypes = [u16p, i64, i64, i64, u16p]
     L.orc_dequantize.restype = None
     L.orc_dequantize.argtypes = [u8p, u8p, f32p, i64, i64, f64p]
     L.orc_sf_mma_bytes.restype = i64
@@ -156,6 +160,21 @@ def quantize(x_bits: np.ndarray, g_row: np.ndarray):
     if rc != 0:
         raise ValueError("columns must be a multiple of 16")
     return codes, sf
+
+
+def silu_mul(g: float, u: float) -> float:
+    """silu(g) * u in the path's binary32 operation sequence (before the bf16 rounding)."""
+    return float(_load().orc_silu_mul(np.float32(g), np.float32(u)))
+
+
+def swiglu_bf16(gate_up_bits: np.ndarray) -> np.ndarray:
+    """bf16 [R, 2I] (gate | up) -> h = bf16(silu(gate) * up), bf16 bit patterns [R, I]."""
+    gu = _c(gate_up_bits, np.uint16)
+    R, two_i = gu.shape
+    assert two_i % 2 == 0
+    h = np.empty((R, two_i // 2), np.uint16)
+    _load().orc_swiglu_bf16(_p(gu), R, two_i // 2, two_i, _p(h))
+    return h
 
 
 def dequantize(codes: np.ndarray, sf: np.ndarray, g_row: np.ndarray) -> np.ndarray:

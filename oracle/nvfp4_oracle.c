@@ -176,6 +176,57 @@ int orc_quantize(const uint16_t* x, int64_t rows, int64_t cols, int64_t ld,
     return 0;
 }
 
+/* ------------------------------------------------------------------------- */
+/* Producer fusion for the MLP: h = silu(gate) * up, rounded to bf16, is what  */
+/* the down projection quantizes.  The paper fixes no arithmetic for it (the   */
+/* activation is upstream of the quantized linears), so the contract is this   */
+/* binary32 sequence, every step one IEEE operation (fmaf = fused, exact):     */
+/*   t = clamp(-g, -87, 87)                                                    */
+/*   z = t * log2(e);  n = rint(z);  r = fmaf(t, log2(e), -n)     r in [-.5,.5] */
+/*   p = 2^r by a degree-5 polynomial (Horner, fmaf);  e = p * 2^n             */
+/*   s = g * (1 / (1 + e));   h = bf16_rne(s * u)                              */
+/* ------------------------------------------------------------------------- */
+static inline float orc_exp_poly(float t) {
+    const float LOG2E = 1.44269504088896341f;
+    if (t < -87.0f) t = -87.0f;
+    if (t > 87.0f) t = 87.0f;
+    const float z = t * LOG2E;
+    const float n = rintf(z);
+    const float r = fmaf(t, LOG2E, -n);
+    float p = 1.3333558146e-3f;                 /* ln2^5/120 and friends */
+    p = fmaf(p, r, 9.6181291076e-3f);
+    p = fmaf(p, r, 5.5504108665e-2f);
+    p = fmaf(p, r, 2.4022650696e-1f);
+    p = fmaf(p, r, 6.9314718056e-1f);
+    p = fmaf(p, r, 1.0f);
+    union { float f; uint32_t u; } sc;
+    sc.u = (uint32_t)((int32_t)n + 127) << 23;  /* 2^n, n in [-126, 126] after the clamp */
+    return p * sc.f;
+}
+
+float orc_silu_mul(float g, float u) {
+    const float e = orc_exp_poly(-g);
+    const float s = g * (1.0f / (1.0f + e));
+    return s * u;
+}
+
+static inline uint16_t orc_f32_to_bf16(float f) {
+    uint32_t b;
+    memcpy(&b, &f, 4);
+    if ((b & 0x7FFFFFFFu) > 0x7F800000u) return 0x7FC0;
+    return (uint16_t)((b + 0x7FFFu + ((b >> 16) & 1u)) >> 16);
+}
+
+/* gate_up: bf16 [rows, 2*inner] (gate in columns [0, inner), up in [inner, 2*inner)), row */
+/* stride ld; h: bf16 [rows, inner].                                                        */
+void orc_swiglu_bf16(const uint16_t* gate_up, int64_t rows, int64_t inner, int64_t ld, uint16_t* h) {
+    #pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t c = 0; c < inner; ++c)
+            h[r * inner + c] = orc_f32_to_bf16(orc_silu_mul(bf16_to_f32(gate_up[r * ld + c]),
+                                                            bf16_to_f32(gate_up[r * ld + inner + c])));
+}
+
 /* x_hat = e2m1(code) * e4m3(scale) * g, evaluated in double (every factor is a
  * binary32 with few significant bits, so the double product is exact). */
 void orc_dequantize(const uint8_t* codes, const uint8_t* sf, const float* g_row,

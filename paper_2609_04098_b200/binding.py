@@ -23,7 +23,7 @@ OUT_F32 = 1
 MAX_SEGMENTS = 32
 
 EXPORTS = (
-    "nvfp4_sf_bytes", "nvfp4_calibrate", "nvfp4_quantize_act", "nvfp4_quantize_weight",
+    "nvfp4_sf_bytes", "nvfp4_calibrate", "nvfp4_quantize_act", "nvfp4_swiglu_quantize", "nvfp4_quantize_weight",
     "nvfp4_linear", "nvfp4_linear_workspace_bytes", "nvfp4_linear_bf16",
     "nvfp4_linear_bf16_workspace_bytes", "nvfp4_linear_bf16_static", "nvfp4_static_status", "nvfp4_workspace_reset", "nvfp4_device_status",
     "nvfp4_launch_count", "nvfp4_set_gemm_variant", "nvfp4_gemm_variants", "nvfp4_status_string",
@@ -59,6 +59,8 @@ def lib() -> ctypes.CDLL:
     L.nvfp4_calibrate.argtypes = [vp, i64, i64, i64, vp, vp, vp]
     L.nvfp4_quantize_act.restype = i32
     L.nvfp4_quantize_act.argtypes = [vp, i64, i64, i64, vp, vp, vp, i32, vp]
+    L.nvfp4_swiglu_quantize.restype = i32
+    L.nvfp4_swiglu_quantize.argtypes = [vp, i64, i64, i64, vp, vp, vp, i32, vp]
     L.nvfp4_quantize_weight.restype = i32
     L.nvfp4_quantize_weight.argtypes = [vp, i64, i64, i64, segp, i32, vp, i32, vp, vp, i32, vp]
     L.nvfp4_linear.restype = i32
@@ -155,6 +157,17 @@ def nvfp4_quantize_act(x: torch.Tensor, g: torch.Tensor, layout: int = SF_MMA, o
     codes, sf = out if out is not None else alloc_quantized(M, K, x.device, layout)
     _check(lib().nvfp4_quantize_act(_ptr(x), M, K, x.stride(0), _ptr(g), _ptr(codes), _ptr(sf), layout,
                                     _stream(stream)), "nvfp4_quantize_act")
+    return codes, sf
+
+
+def nvfp4_swiglu_quantize(gate_up: torch.Tensor, g: torch.Tensor, layout: int = SF_MMA, out=None, stream=None):
+    """bf16 [M, 2I] (gate | up) -> NVFP4 of bf16(silu(gate) * up): (codes u8 [M, I/2], scale bytes)."""
+    assert gate_up.is_cuda and gate_up.dtype == torch.bfloat16 and gate_up.dim() == 2 and gate_up.stride(1) == 1
+    M, two_i = gate_up.shape
+    inner = two_i // 2
+    codes, sf = out if out is not None else alloc_quantized(M, inner, gate_up.device, layout)
+    _check(lib().nvfp4_swiglu_quantize(_ptr(gate_up), M, inner, gate_up.stride(0), _ptr(g), _ptr(codes), _ptr(sf),
+                                       layout, _stream(stream)), "nvfp4_swiglu_quantize")
     return codes, sf
 
 

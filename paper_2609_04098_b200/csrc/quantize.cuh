@@ -116,10 +116,44 @@ __device__ __forceinline__ uint2 quantize_block(const uint32_t (&v)[8], float g,
     return out;
 }
 
+// silu(g) * u in the binary32 sequence that the path fixes for the MLP's activation (each step
+// one IEEE operation, fmaf fused):  t = clamp(-g, -87, 87);  n = rint(t * log2 e);
+// r = fmaf(t, log2 e, -n);  2^r by a degree-5 polynomial;  e = 2^r * 2^n;
+// s = g * (1 / (1 + e));  result s * u.
+__device__ __forceinline__ float silu_mul(float g, float u) {
+    const float LOG2E = 1.44269504088896341f;
+    float t = -g;
+    if (t < -87.0f) t = -87.0f;
+    if (t > 87.0f) t = 87.0f;
+    const float n = rintf(__fmul_rn(t, LOG2E));
+    const float r = __fmaf_rn(t, LOG2E, -n);
+    float p = 1.3333558146e-3f;
+    p = __fmaf_rn(p, r, 9.6181291076e-3f);
+    p = __fmaf_rn(p, r, 5.5504108665e-2f);
+    p = __fmaf_rn(p, r, 2.4022650696e-1f);
+    p = __fmaf_rn(p, r, 6.9314718056e-1f);
+    p = __fmaf_rn(p, r, 1.0f);
+    const float e = __fmul_rn(p, __int_as_float((static_cast<int>(n) + 127) << 23));
+    const float s = __fmul_rn(g, __frcp_rn(__fadd_rn(1.0f, e)));
+    return __fmul_rn(s, u);
+}
+
+// 16 gate values and 16 up values (packed bf16) -> 16 values of bf16(silu(gate) * up), packed
+__device__ __forceinline__ void swiglu_block(const uint32_t (&g)[8], const uint32_t (&u)[8], uint32_t (&h)[8]) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const float lo = silu_mul(__uint_as_float(g[i] << 16), __uint_as_float(u[i] << 16));
+        const float hi = silu_mul(__uint_as_float(g[i] & 0xFFFF0000u), __uint_as_float(u[i] & 0xFFFF0000u));
+        __nv_bfloat162 b2 = __floats2bfloat162_rn(lo, hi);
+        h[i] = *reinterpret_cast<uint32_t*>(&b2);
+    }
+}
+
 // A warp owns `chunks_per_unit` consecutive 512-element chunks of one row (a "unit"); units are
 // dealt round-robin to a persistent grid.
-template <bool MMA_LAYOUT, int UNROLL>
-__global__ void __launch_bounds__(256, 5)
+// SWIGLU: x is [M, 2K] (gate | up) and the tensor that is quantized is bf16(silu(gate) * up), [M, K].
+template <bool MMA_LAYOUT, int UNROLL, bool SWIGLU>
+__global__ void __launch_bounds__(256, SWIGLU ? 4 : 5)
 quantize_kernel(const uint16_t* __restrict__ x, int32_t M, int32_t K, int64_t ld,
                 const float* __restrict__ g_ptr, SegTable segs,
                 uint8_t* __restrict__ codes, uint8_t* __restrict__ sf,
@@ -156,6 +190,13 @@ quantize_kernel(const uint16_t* __restrict__ x, int32_t M, int32_t K, int64_t ld
                 col[u] = (c0 + u < c_end) ? (c0 + u) * 512 + lane * 16 : K;
                 if (col[u] < K) {
                     ldg256_stream(xrow + col[u], v[u]);
+                    if (SWIGLU) {
+                        uint32_t up[8], h[8];
+                        ldg256_stream(xrow + K + col[u], up);
+                        swiglu_block(v[u], up, h);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) v[u][i] = h[i];
+                    }
                 } else {
 #pragma unroll
                     for (int i = 0; i < 8; ++i) v[u][i] = 0u;

@@ -122,3 +122,56 @@ def test_gdn_weight_full_size():
     codes_o, sf_o, g_o, _ = gu.oracle_quantized(w, segments=segs)
     assert np.array_equal(g_d.cpu().numpy(), g_o)
     gu.check_quantized(codes_d, sf_d, nv.SF_MMA, codes_o, sf_o, synth.HIDDEN)
+
+
+# ---- producer fusion: silu(gate) * up -> quantize in one pass -------------------------------
+def _swiglu_case(M, inner, layout=nv.SF_MMA, seed=9, ld_pad=0):
+    segs = synth.make_segments((("gate", M, 1.0),))
+    gu = synth.weights(seed, 60, segs, 2 * inner)                 # bf16 [M, 2*inner] ~ N(0, 1): gate | up
+    # a few hot entries, as after a projection of outlier channels
+    gu[:, 7] = synth.f64_to_bf16_bits(synth.bf16_bits_to_f32(gu[:, 7]).astype(np.float64) * 12.0)
+    h = oracle.swiglu_bf16(gu)
+    _, g = oracle.calibrate(h)
+    t = synth.to_torch_bf16(gu).to(gu_mod.DEV)
+    if ld_pad:
+        buf = torch.zeros((M, 2 * inner + ld_pad), dtype=torch.bfloat16, device=gu_mod.DEV)
+        buf[:, :2 * inner] = t
+        t = buf[:, :2 * inner]
+    codes_d, sf_d = nv.nvfp4_swiglu_quantize(t, gu_mod.dev_f32(g), layout)
+    torch.cuda.synchronize()
+    codes_o, sf_o, _, _ = gu_mod.oracle_quantized(h, g=g)
+    gu_mod.check_quantized(codes_d, sf_d, layout, codes_o, sf_o, inner)
+    return t, g, codes_d, sf_d
+
+
+from tests import gpu_util as gu_mod  # noqa: E402  (alias: `gu` above is the helper module too)
+
+
+@pytest.mark.parametrize("M,inner", [(1, 16), (5, 48), (128, 512), (130, 1040), (300, 17408 // 4)])
+@pytest.mark.parametrize("layout", [nv.SF_MMA, nv.SF_LINEAR])
+def test_swiglu_quantize_matches_oracle_composition(M, inner, layout):
+    _swiglu_case(M, inner, layout)
+
+
+def test_swiglu_quantize_strided_and_equal_to_unfused_path():
+    t, g, codes_d, sf_d = _swiglu_case(96, 2048, ld_pad=64)
+    # the same result as materialising h in bf16 and calling nvfp4_quantize_act on it
+    gu_host = gu_mod.host_bits(t.contiguous())
+    h = gu_mod.dev_bf16(oracle.swiglu_bf16(gu_host))
+    c2, s2 = nv.nvfp4_quantize_act(h, gu_mod.dev_f32(g))
+    torch.cuda.synchronize()
+    assert torch.equal(c2, codes_d) and torch.equal(s2, sf_d)
+
+
+def test_swiglu_extreme_gates():
+    M, inner = 4, 64
+    vals = np.zeros((M, 2 * inner))
+    vals[:, :inner] = np.linspace(-120, 120, inner)[None, :] * np.array([1.0, 0.5, 0.01, -1.0])[:, None]
+    vals[:, inner:] = np.array([1.0, -3.0, 250.0, 0.125])[:, None]
+    gu = synth.f64_to_bf16_bits(vals).reshape(M, 2 * inner)
+    h = oracle.swiglu_bf16(gu)
+    _, g = oracle.calibrate(h)
+    codes_d, sf_d = nv.nvfp4_swiglu_quantize(gu_mod.dev_bf16(gu), gu_mod.dev_f32(g))
+    torch.cuda.synchronize()
+    codes_o, sf_o, _, _ = gu_mod.oracle_quantized(h, g=g)
+    gu_mod.check_quantized(codes_d, sf_d, nv.SF_MMA, codes_o, sf_o, inner)
