@@ -75,9 +75,12 @@ __device__ __forceinline__ void ldg256_stream(const void* p, uint32_t (&v)[8]) {
                  : "l"(p));
 }
 
+// per 16-bit half: magnitude = max(|a|, |b|) (the sign bit of the result is sign(a) xor sign(b)
+// and is masked off by the caller)
 __device__ __forceinline__ uint32_t bf16x2_absmax(uint32_t a, uint32_t b) {
-    __nv_bfloat162 r = __hmax2(*reinterpret_cast<__nv_bfloat162*>(&a), *reinterpret_cast<__nv_bfloat162*>(&b));
-    return *reinterpret_cast<uint32_t*>(&r);
+    uint32_t r;
+    asm("max.xorsign.abs.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
 }
 
 // One 16-element block held by one lane: returns the 16 packed codes (element i in nibble i)
@@ -86,11 +89,9 @@ __device__ __forceinline__ uint32_t bf16x2_absmax(uint32_t a, uint32_t b) {
 //     s8 = e4m3(bmax * c1),  c1 = 1 / (6 g);   code = e2m1(x * (1 / (e4m3(s8) * g)))
 __device__ __forceinline__ uint2 quantize_block(const uint32_t (&v)[8], float g, float c1, uint32_t& s8_out) {
     // block maximum on packed bf16 pairs (|x| is a bit mask; the maximum of bf16 values is exact)
-    uint32_t m = bf16x2_absmax(v[0] & 0x7FFF7FFFu, v[1] & 0x7FFF7FFFu);
-    m = bf16x2_absmax(m, bf16x2_absmax(v[2] & 0x7FFF7FFFu, v[3] & 0x7FFF7FFFu));
-    uint32_t m2 = bf16x2_absmax(v[4] & 0x7FFF7FFFu, v[5] & 0x7FFF7FFFu);
-    m2 = bf16x2_absmax(m2, bf16x2_absmax(v[6] & 0x7FFF7FFFu, v[7] & 0x7FFF7FFFu));
-    m = bf16x2_absmax(m, m2);
+    uint32_t m = bf16x2_absmax(bf16x2_absmax(v[0], v[1]), bf16x2_absmax(v[2], v[3]));
+    const uint32_t m2 = bf16x2_absmax(bf16x2_absmax(v[4], v[5]), bf16x2_absmax(v[6], v[7]));
+    m = bf16x2_absmax(m, m2) & 0x7FFF7FFFu;
     const float bmax = fmaxf(__uint_as_float(m << 16), __uint_as_float(m & 0xFFFF0000u));
     const uint32_t s8 = f32_to_e4m3(__fmul_rn(bmax, c1));
     s8_out = s8;
@@ -122,9 +123,7 @@ __device__ __forceinline__ uint2 quantize_block(const uint32_t (&v)[8], float g,
 // s = g * (1 / (1 + e));  result s * u.
 __device__ __forceinline__ float silu_mul(float g, float u) {
     const float LOG2E = 1.44269504088896341f;
-    float t = -g;
-    if (t < -87.0f) t = -87.0f;
-    if (t > 87.0f) t = 87.0f;
+    const float t = fminf(fmaxf(-g, -87.0f), 87.0f);
     const float n = rintf(__fmul_rn(t, LOG2E));
     const float r = __fmaf_rn(t, LOG2E, -n);
     float p = 1.3333558146e-3f;
@@ -166,9 +165,12 @@ quantize_kernel(const uint16_t* __restrict__ x, int32_t M, int32_t K, int64_t ld
     const float g_single = (segs.nseg == 0) ? __ldg(g_ptr) : 0.0f;
     const float c1_single = __fdiv_rn(1.0f, __fmul_rn(6.0f, g_single));
 
-    for (int32_t unit = warp_global; unit < total_units; unit += nwarps) {
-        const int32_t row = unit / units_per_row;                  // one division per >= 512 elements
-        const int32_t c_begin = (unit - row * units_per_row) * chunks_per_unit;
+    // (row, part) of this warp's unit, advanced without a division per unit
+    int32_t row = warp_global / units_per_row, part = warp_global - row * units_per_row;
+    const int32_t d_row = nwarps / units_per_row, d_part = nwarps - d_row * units_per_row;
+    for (int32_t unit = warp_global; unit < total_units; unit += nwarps, row += d_row, part += d_part) {
+        if (part >= units_per_row) { part -= units_per_row; ++row; }
+        const int32_t c_begin = part * chunks_per_unit;
         const int32_t c_end = min(chunks_per_row, c_begin + chunks_per_unit);
         float g = g_single, c1 = c1_single;
         if (segs.nseg != 0) {
