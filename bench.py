@@ -176,16 +176,15 @@ def run_gpu(args):
     from paper_2609_04098_b200 import binding as nv
     from paper_2609_04098_b200 import build as nvbuild
 
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
+    from paper_2609_04098_b200.replicas import Replicas
+
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
+    reps = Replicas(backend="nccl", device=dev)          # independent replicas: barrier + max only
+    rank, world = reps.rank, reps.world
     nvbuild.build()
     nv.lib()
     if args.variant:
@@ -278,10 +277,7 @@ def run_gpu(args):
     else:
         raise SystemExit("unknown workload")
 
-    def barrier():
-        if world > 1:
-            import torch.distributed as dist
-            dist.barrier()
+    barrier = reps.barrier
 
     # ---- device-resident timing
     for _ in range(max(3, args.warmup)):
@@ -303,12 +299,7 @@ def run_gpu(args):
     barrier()
     clocks = sampler.stop()
     launches = nv.launch_count() - launches0
-    total_ms = t_start.elapsed_time(t_end)
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([total_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = reps.max_over_ranks(t_start.elapsed_time(t_end))
     ms_per_step = total_ms / args.steps
     value = wl.flops * world / (ms_per_step * 1e-3) / 1e12
 
@@ -432,12 +423,7 @@ def run_gpu(args):
         e2e_step()
     s1.record(stream)
     torch.cuda.synchronize()
-    e2e_ms = s0.elapsed_time(s1) / e2e_steps
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([e2e_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = reps.max_over_ranks(s0.elapsed_time(s1) / e2e_steps)
     result["e2e"] = {"value": round(wl.flops * world / (e2e_ms * 1e-3) / 1e12, 2), "unit": "TFLOP/s",
                      "ms_per_step": round(e2e_ms, 3), "h2d_bytes_per_step": h2d_bytes,
                      "d2h_bytes_per_step": d2h_bytes}
@@ -460,9 +446,7 @@ def run_gpu(args):
                 "gpu_launches": int(launches), "clocks": clocks}
         line.update(result)
         print(json.dumps(line))
-    if world > 1:
-        import torch.distributed as dist
-        dist.destroy_process_group()
+    reps.close()
 
 
 # --------------------------------------------------------------------------- CPU oracle arm
