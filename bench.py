@@ -183,8 +183,8 @@ def run_gpu(args):
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    reps = Replicas(backend="nccl", device=dev)          # independent replicas: barrier + max only
-    rank, world = reps.rank, reps.world
+    group = Replicas(backend="nccl", device=dev)         # independent replicas: barrier + max only
+    rank, world = group.rank, group.world
     nvbuild.build()
     nv.lib()
     if args.variant:
@@ -277,7 +277,7 @@ def run_gpu(args):
     else:
         raise SystemExit("unknown workload")
 
-    barrier = reps.barrier
+    barrier = group.barrier
 
     # ---- device-resident timing
     for _ in range(max(3, args.warmup)):
@@ -299,7 +299,7 @@ def run_gpu(args):
     barrier()
     clocks = sampler.stop()
     launches = nv.launch_count() - launches0
-    total_ms = reps.max_over_ranks(t_start.elapsed_time(t_end))
+    total_ms = group.max_over_ranks(t_start.elapsed_time(t_end))
     ms_per_step = total_ms / args.steps
     value = wl.flops * world / (ms_per_step * 1e-3) / 1e12
 
@@ -423,7 +423,7 @@ def run_gpu(args):
         e2e_step()
     s1.record(stream)
     torch.cuda.synchronize()
-    e2e_ms = reps.max_over_ranks(s0.elapsed_time(s1) / e2e_steps)
+    e2e_ms = group.max_over_ranks(s0.elapsed_time(s1) / e2e_steps)
     result["e2e"] = {"value": round(wl.flops * world / (e2e_ms * 1e-3) / 1e12, 2), "unit": "TFLOP/s",
                      "ms_per_step": round(e2e_ms, 3), "h2d_bytes_per_step": h2d_bytes,
                      "d2h_bytes_per_step": d2h_bytes}
@@ -446,7 +446,7 @@ def run_gpu(args):
                 "gpu_launches": int(launches), "clocks": clocks}
         line.update(result)
         print(json.dumps(line))
-    reps.close()
+    group.close()
 
 
 # --------------------------------------------------------------------------- CPU oracle arm
