@@ -224,6 +224,23 @@ nvfp4_status nvfp4_workspace_reset(void* d_workspace, size_t workspace_bytes, vo
  */
 nvfp4_status nvfp4_device_status(const void* d_workspace, void* stream);
 
+/*
+ * Time limit of every wait inside the GEMM kernel, in nanoseconds (0 restores the default of
+ * 2 s).  A CTA whose wait runs out stops issuing work, lets what it has in flight finish, frees
+ * its tensor memory and raises NVFP4_ERR_TIMEOUT in the workspace status word; the kernel
+ * returns and the CUDA context stays usable.  Process-wide.  A limit shorter than a memory
+ * round trip makes a correct launch give up, which is how the failure path is tested.
+ */
+nvfp4_status nvfp4_set_wait_limit_ns(uint64_t limit_ns);
+
+/*
+ * Failure-path self-test: one CTA waits, with the same bounded wait the GEMM uses, on a barrier
+ * that nothing ever completes, for at most limit_ns (1 .. 1e9), then writes NVFP4_ERR_TIMEOUT to
+ * the workspace status word and returns normally.  Read the result with nvfp4_device_status.
+ */
+nvfp4_status nvfp4_selftest_bounded_wait(void* d_workspace, size_t workspace_bytes, uint64_t limit_ns,
+                                         void* stream);
+
 /* Number of this library's kernel launches enqueued so far by this process. */
 uint64_t nvfp4_launch_count(void);
 

@@ -26,7 +26,7 @@ EXPORTS = (
     "nvfp4_sf_bytes", "nvfp4_calibrate", "nvfp4_quantize_act", "nvfp4_swiglu_quantize", "nvfp4_quantize_weight",
     "nvfp4_linear", "nvfp4_linear_workspace_bytes", "nvfp4_linear_bf16",
     "nvfp4_linear_bf16_workspace_bytes", "nvfp4_linear_bf16_static", "nvfp4_static_status", "nvfp4_workspace_reset", "nvfp4_device_status",
-    "nvfp4_launch_count", "nvfp4_set_gemm_variant", "nvfp4_gemm_variants", "nvfp4_status_string",
+    "nvfp4_set_wait_limit_ns", "nvfp4_selftest_bounded_wait", "nvfp4_launch_count", "nvfp4_set_gemm_variant", "nvfp4_gemm_variants", "nvfp4_status_string",
 )
 
 
@@ -79,6 +79,10 @@ def lib() -> ctypes.CDLL:
     L.nvfp4_workspace_reset.argtypes = [vp, sz, vp]
     L.nvfp4_device_status.restype = i32
     L.nvfp4_device_status.argtypes = [vp, vp]
+    L.nvfp4_set_wait_limit_ns.restype = i32
+    L.nvfp4_set_wait_limit_ns.argtypes = [ctypes.c_uint64]
+    L.nvfp4_selftest_bounded_wait.restype = i32
+    L.nvfp4_selftest_bounded_wait.argtypes = [vp, sz, ctypes.c_uint64, vp]
     L.nvfp4_launch_count.restype = ctypes.c_uint64
     L.nvfp4_launch_count.argtypes = []
     L.nvfp4_set_gemm_variant.restype = i32
@@ -127,6 +131,17 @@ def launch_count() -> int:
 
 def set_gemm_variant(variant: int) -> None:
     _check(lib().nvfp4_set_gemm_variant(int(variant)), "nvfp4_set_gemm_variant")
+
+
+def set_wait_limit_ns(limit_ns: int) -> None:
+    """Limit of every in-kernel wait of the GEMM (0 = default 2 s)."""
+    _check(lib().nvfp4_set_wait_limit_ns(int(limit_ns)), "nvfp4_set_wait_limit_ns")
+
+
+def selftest_bounded_wait(workspace: torch.Tensor, limit_ns: int, stream=None) -> None:
+    """Enqueue the failure-path self-test (a wait that nothing completes); read device_status after."""
+    _check(lib().nvfp4_selftest_bounded_wait(_ptr(workspace), workspace.numel(), int(limit_ns), _stream(stream)),
+           "nvfp4_selftest_bounded_wait")
 
 
 def sf_bytes(rows: int, K: int, layout: int = SF_MMA) -> int:

@@ -464,6 +464,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     }
 
     // ---------------------------------------------------------------- teardown
+    // a CTA that gave up may still have copies and MMAs in flight (its own or its partner's,
+    // which signal this CTA's barriers): give them time to land before anything is torn down
+    if (*abort_flag != 0u) __nanosleep(50000);
     ptx::tc_fence_before();
     if (PAIR) ptx::cluster_sync_all(); else __syncthreads();   // nobody touches TMEM or a partner's barriers after this
     if (warp == 6) {

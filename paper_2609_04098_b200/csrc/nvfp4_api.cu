@@ -20,6 +20,7 @@ namespace {
 
 std::atomic<uint64_t> g_launches{0};
 std::atomic<int> g_variant{0};
+std::atomic<uint64_t> g_wait_limit_ns{0};          // 0 = default
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // every in-kernel wait gives up after 2 s
 
 inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
@@ -490,7 +491,10 @@ nvfp4_status nvfp4_linear(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const
     p.flags = flags;
     p.nseg = nseg;
     for (int i = 0; i < nseg; ++i) p.seg_end[i] = static_cast<int32_t>(segs[i].col_begin + segs[i].col_count);
-    p.wait_limit_ns = kWaitLimitNs;
+    {
+        const uint64_t lim = g_wait_limit_ns.load(std::memory_order_relaxed);
+        p.wait_limit_ns = lim != 0 ? lim : kWaitLimitNs;
+    }
 #ifdef NVFP4_PROBE
     p.probe = getenv("NVFP4_PROBE") ? static_cast<uint32_t>(atoi(getenv("NVFP4_PROBE"))) : 0u;
     p.trace = getenv("NVFP4_TRACE_PTR") ? reinterpret_cast<unsigned long long*>(strtoull(getenv("NVFP4_TRACE_PTR"), nullptr, 16)) : nullptr;
@@ -584,6 +588,41 @@ nvfp4_status nvfp4_device_status(const void* d_workspace, void* stream) {
         return NVFP4_ERR_CUDA;
     if (cudaStreamSynchronize(as_stream(stream)) != cudaSuccess) return NVFP4_ERR_CUDA;
     return word == 0u ? NVFP4_OK : (word == NVFP4_ERR_TIMEOUT ? NVFP4_ERR_TIMEOUT : NVFP4_ERR_CUDA);
+}
+
+namespace nvfp4 {
+// One CTA waits, with the library's bounded wait, on a barrier that nothing ever completes.
+__global__ void bounded_wait_selftest_kernel(uint32_t* status, uint64_t limit_ns) {
+    __shared__ uint64_t bar;
+    __shared__ uint32_t abort_flag;
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(&bar, 1);
+        abort_flag = 0u;
+        ptx::fence_barrier_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const bool completed = ptx::mbar_wait_bounded(&bar, 0u, &abort_flag, limit_ns);
+        *status = completed ? static_cast<uint32_t>(NVFP4_OK) : static_cast<uint32_t>(NVFP4_ERR_TIMEOUT);
+    }
+}
+}  // namespace nvfp4
+
+nvfp4_status nvfp4_selftest_bounded_wait(void* d_workspace, size_t workspace_bytes, uint64_t limit_ns, void* stream) {
+    if (d_workspace == nullptr) return NVFP4_ERR_NULL;
+    if (workspace_bytes < kStatusBytes) return NVFP4_ERR_WORKSPACE;
+    if (limit_ns == 0 || limit_ns > 1000000000ull) return NVFP4_ERR_SHAPE;      // at most one second
+    DeviceInfo info;
+    nvfp4_status st = check_arch(info);
+    if (st != NVFP4_OK) return st;
+    bounded_wait_selftest_kernel<<<1, 32, 0, as_stream(stream)>>>(reinterpret_cast<uint32_t*>(d_workspace), limit_ns);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+}
+
+nvfp4_status nvfp4_set_wait_limit_ns(uint64_t limit_ns) {
+    g_wait_limit_ns.store(limit_ns, std::memory_order_relaxed);
+    return NVFP4_OK;
 }
 
 uint64_t nvfp4_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }

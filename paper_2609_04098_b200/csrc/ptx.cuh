@@ -61,7 +61,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 
-// Bounded wait: spins on try_wait; every 256 failed polls it looks at the CTA's
+// Bounded wait: spins on try_wait; every 32 failed polls it looks at the CTA's
 // abort flag and at the wall clock.  Returns false (and raises the abort flag) if
 // `limit_ns` passes or another role already gave up, so no wait can hang the GPU.
 // `peer_abort` (0 = none) is the cluster address of the partner CTA's abort flag: a CTA
@@ -72,16 +72,14 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
                                                   volatile uint32_t* abort_flag, uint64_t limit_ns,
                                                   uint32_t peer_abort = 0u, uint32_t backoff_ns = 0u) {
     if (mbar_try_wait(bar, parity)) return true;
-    uint64_t t0 = 0;
+    const uint64_t t0 = globaltimer_ns();
     uint32_t polls = 0;
     while (true) {
         if (backoff_ns != 0u) __nanosleep(backoff_ns);
         if (mbar_try_wait(bar, parity)) return true;
-        if ((++polls & 255u) == 0u) {
+        if ((++polls & 31u) == 0u) {
             if (*abort_flag != 0u) return false;
-            uint64_t now = globaltimer_ns();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > limit_ns) {
+            if (globaltimer_ns() - t0 > limit_ns) {
                 *abort_flag = 1u;
                 if (peer_abort != 0u) asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(peer_abort), "r"(1u) : "memory");
                 return false;
