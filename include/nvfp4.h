@@ -137,6 +137,23 @@ nvfp4_status nvfp4_quantize_weight(const void* d_w, int64_t N, int64_t K, int64_
                                    nvfp4_sf_layout layout, void* stream);
 
 /*
+ * Checkpoint-side repair (paper: Section 6 -- "rewrite each fused group to the shared global
+ * scale and fold the ratio into the per-block E4M3 scales", re-rounding error <= 6.2 %): lets a
+ * GEMM with ONE global scale serve a fused group whose modules were calibrated separately.
+ *     g* = max_j g_seg[j];   s'_b = e4m3_rne_sat( e4m3(s_b) * (g_seg[j] / g*) )   (binary32)
+ * Codes are unchanged.  Afterwards nvfp4_linear with the single segment [0, N) and g* reproduces
+ * the per-module result up to the re-rounding of the scales; the per-segment epilogue of
+ * nvfp4_linear remains the exact form of the repair.
+ *   d_sf_in / d_sf_out  scale bytes of the [N, K] weight in `layout` (may be the same buffer)
+ *   segs, d_g_seg       the modules and their calibrated scales (segs: host array)
+ *   d_g_shared          out: g* (device scalar)
+ * Errors: NULL, shape, layout, NVFP4_ERR_SEGMENTS, misaligned scale pointers.
+ */
+nvfp4_status nvfp4_harmonize_scales(const uint8_t* d_sf_in, int64_t N, int64_t K, nvfp4_sf_layout layout,
+                                    const nvfp4_segment* segs, const float* d_g_seg, int nseg,
+                                    uint8_t* d_sf_out, float* d_g_shared, void* stream);
+
+/*
  * The W4A4 linear layer (paper: Background, "NVFP4": the GEMM runs on 4-bit tensor
  * cores; Section 6: per-module global scales meeting in one fused GEMM -- here each
  * segment of output columns gets its own global scale in the epilogue, which is

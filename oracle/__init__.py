@@ -68,6 +68,8 @@ def _load():
     L.orc_swiglu_bf16.argtypes = [u16p, i64, i64, i64, u16p]
     L.orc_dequantize.restype = None
     L.orc_dequantize.argtypes = [u8p, u8p, f32p, i64, i64, f64p]
+    L.orc_harmonize_scales.restype = ctypes.c_float
+    L.orc_harmonize_scales.argtypes = [u8p, i64, i64, f32p, u8p]
     L.orc_sf_mma_bytes.restype = i64
     L.orc_sf_mma_bytes.argtypes = [i64, i64]
     L.orc_sf_mma_index.restype = i64
@@ -184,6 +186,15 @@ def dequantize(codes: np.ndarray, sf: np.ndarray, g_row: np.ndarray) -> np.ndarr
     out = np.empty((R, C), np.float64)
     _load().orc_dequantize(_p(codes), _p(sf), _p(_c(g_row, np.float32)), R, C, _p(out))
     return out
+
+
+def harmonize_scales(sf_linear: np.ndarray, g_row: np.ndarray):
+    """Shared global scale for a fused group: returns (re-rounded scale bytes, g* = max g)."""
+    sf = _c(sf_linear, np.uint8)
+    g_row = _c(g_row, np.float32)
+    out = np.empty_like(sf)
+    gstar = _load().orc_harmonize_scales(_p(sf), sf.shape[0], sf.shape[1], _p(g_row), _p(out))
+    return out, np.float32(gstar)
 
 
 def sf_mma_bytes(rows: int, cols: int) -> int:

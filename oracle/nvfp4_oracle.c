@@ -243,6 +243,28 @@ void orc_dequantize(const uint8_t* codes, const uint8_t* sf, const float* g_row,
 }
 
 /* ------------------------------------------------------------------------- */
+/* Checkpoint-side repair of Section 6: give a fused group ONE global scale    */
+/* (the maximum of its modules' scales) and fold each module's ratio into its  */
+/* E4M3 block scales, re-rounding them:                                        */
+/*     g* = max_j g_j ;  r_j = g_j / g*  (f32 divide) ;                        */
+/*     s'_b = e4m3_rne_sat( e4m3(s_b) * r_j )   (f32 multiply)                 */
+/* Codes are untouched.  sf / sf_out: [rows, nb] row-major; g_row[r] is the    */
+/* scale of the module that row r belongs to.                                  */
+/* ------------------------------------------------------------------------- */
+float orc_harmonize_scales(const uint8_t* sf, int64_t rows, int64_t nb, const float* g_row, uint8_t* sf_out) {
+    float gstar = 0.0f;
+    for (int64_t r = 0; r < rows; ++r)
+        if (g_row[r] > gstar) gstar = g_row[r];
+    #pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r) {
+        const float ratio = g_row[r] / gstar;                              /* f32 divide */
+        for (int64_t b = 0; b < nb; ++b)
+            sf_out[r * nb + b] = orc_e4m3_encode(orc_e4m3_decode(sf[r * nb + b]) * ratio);   /* f32 multiply */
+    }
+    return gstar;
+}
+
+/* ------------------------------------------------------------------------- */
 /* Scale-byte storage order the block-scaled tensor-core instruction reads:   */
 /* 128 rows x 4 blocks form one 512-byte atom; atoms of one 128-row band are  */
 /* contiguous along K; rows padded to 128, blocks to 4, padding bytes zero.   */

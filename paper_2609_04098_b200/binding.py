@@ -24,7 +24,7 @@ MAX_SEGMENTS = 32
 
 EXPORTS = (
     "nvfp4_sf_bytes", "nvfp4_calibrate", "nvfp4_quantize_act", "nvfp4_swiglu_quantize", "nvfp4_quantize_weight",
-    "nvfp4_linear", "nvfp4_linear_workspace_bytes", "nvfp4_linear_bf16",
+    "nvfp4_harmonize_scales", "nvfp4_linear", "nvfp4_linear_workspace_bytes", "nvfp4_linear_bf16",
     "nvfp4_linear_bf16_workspace_bytes", "nvfp4_linear_bf16_static", "nvfp4_static_status", "nvfp4_workspace_reset", "nvfp4_device_status",
     "nvfp4_set_wait_limit_ns", "nvfp4_selftest_bounded_wait", "nvfp4_launch_count", "nvfp4_set_gemm_variant", "nvfp4_gemm_variants", "nvfp4_status_string",
 )
@@ -63,6 +63,8 @@ def lib() -> ctypes.CDLL:
     L.nvfp4_swiglu_quantize.argtypes = [vp, i64, i64, i64, vp, vp, vp, i32, vp]
     L.nvfp4_quantize_weight.restype = i32
     L.nvfp4_quantize_weight.argtypes = [vp, i64, i64, i64, segp, i32, vp, i32, vp, vp, i32, vp]
+    L.nvfp4_harmonize_scales.restype = i32
+    L.nvfp4_harmonize_scales.argtypes = [vp, i64, i64, i32, segp, vp, i32, vp, vp, vp]
     L.nvfp4_linear.restype = i32
     L.nvfp4_linear.argtypes = [vp, vp, vp, i64, i64, vp, vp, i64, segp, vp, i32, vp, i64, u32, vp, sz, vp]
     L.nvfp4_linear_workspace_bytes.restype = sz
@@ -202,6 +204,17 @@ def nvfp4_quantize_weight(w: torch.Tensor, segments, g_seg: Optional[torch.Tenso
                                        calibrate, _ptr(codes), _ptr(sf), layout, _stream(stream)),
            "nvfp4_quantize_weight")
     return codes, sf, g_seg
+
+
+def nvfp4_harmonize_scales(w_sf: torch.Tensor, N: int, K: int, segments, g_seg: torch.Tensor,
+                           layout: int = SF_MMA, stream=None):
+    """Shared global scale for a fused group: returns (re-rounded scale bytes, g* device scalar)."""
+    pairs = seg_pairs(segments)
+    out = torch.empty_like(w_sf)
+    g_shared = torch.empty(1, dtype=torch.float32, device=w_sf.device)
+    _check(lib().nvfp4_harmonize_scales(_ptr(w_sf), N, K, layout, _segments(pairs), _ptr(g_seg), len(pairs),
+                                        _ptr(out), _ptr(g_shared), _stream(stream)), "nvfp4_harmonize_scales")
+    return out, g_shared
 
 
 def alloc_workspace(device, M: int = 0, N: int = 0, K: int = 0, nseg: int = 1, fused: bool = False) -> torch.Tensor:

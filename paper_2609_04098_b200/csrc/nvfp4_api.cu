@@ -427,6 +427,39 @@ nvfp4_status nvfp4_swiglu_quantize(const void* d_gate_up, int64_t M, int64_t inn
     return quantize_impl(d_gate_up, M, inner, ld, d_g, segs, d_codes, d_sf, layout, info, as_stream(stream), true);
 }
 
+nvfp4_status nvfp4_harmonize_scales(const uint8_t* d_sf_in, int64_t N, int64_t K, nvfp4_sf_layout layout,
+                                    const nvfp4_segment* segs, const float* d_g_seg, int nseg, uint8_t* d_sf_out,
+                                    float* d_g_shared, void* stream) {
+    if (d_sf_in == nullptr || d_sf_out == nullptr || d_g_seg == nullptr || d_g_shared == nullptr) return NVFP4_ERR_NULL;
+    if (N < 0 || K <= 0 || (K % 16) != 0 || N >= (1ll << 31) || K >= (1ll << 31)) return NVFP4_ERR_SHAPE;
+    if (layout != NVFP4_SF_LINEAR && layout != NVFP4_SF_MMA) return NVFP4_ERR_LAYOUT;
+    nvfp4_status st = check_segments(segs, nseg, N);
+    if (st != NVFP4_OK) return st;
+    if (layout == NVFP4_SF_MMA && (((reinterpret_cast<uintptr_t>(d_sf_in) | reinterpret_cast<uintptr_t>(d_sf_out)) & 3u) != 0))
+        return NVFP4_ERR_ALIGN;
+    DeviceInfo info;
+    st = check_arch(info);
+    if (st != NVFP4_OK) return st;
+    cudaStream_t s = as_stream(stream);
+    if (layout == NVFP4_SF_MMA && d_sf_out != d_sf_in) {
+        // padding rows and blocks of the output read as zero scales
+        if (cudaMemsetAsync(d_sf_out, 0, nvfp4_sf_bytes(N, K, layout), s) != cudaSuccess) return NVFP4_ERR_CUDA;
+    }
+    SegTable table;
+    std::memset(&table, 0, sizeof(table));
+    table.nseg = nseg;
+    for (int i = 0; i < nseg; ++i) table.row_end[i] = static_cast<int32_t>(segs[i].col_begin + segs[i].col_count);
+    const int64_t words = N * ((K / 16 + 3) / 4);
+    int64_t blocks = (words + 255) / 256;
+    if (blocks > info.sm_count * 8) blocks = info.sm_count * 8;
+    if (blocks < 1) blocks = 1;
+    harmonize_kernel<<<static_cast<int>(blocks), 256, 0, s>>>(d_sf_in, d_sf_out, static_cast<int32_t>(N),
+                                                             static_cast<int32_t>(K / 16), layout == NVFP4_SF_MMA ? 1 : 0,
+                                                             d_g_seg, table, d_g_shared);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+}
+
 size_t nvfp4_linear_workspace_bytes(int64_t, int64_t, int64_t, int) { return kStatusBytes; }
 
 nvfp4_status nvfp4_workspace_reset(void* d_workspace, size_t workspace_bytes, void* stream) {

@@ -229,6 +229,40 @@ quantize_kernel(const uint16_t* __restrict__ x, int32_t M, int32_t K, int64_t ld
     }
 }
 
+// ------------------------------------------------------------------ scale harmonisation
+// Shared global scale for a fused group: g* = max_j g_j; every scale byte of module j becomes
+// e4m3(e4m3(s) * (g_j / g*)).  One thread handles the four scale bytes of one row and one
+// 64-element group (one 32-bit word in either layout).
+__global__ void __launch_bounds__(256)
+harmonize_kernel(const uint8_t* __restrict__ sf_in, uint8_t* __restrict__ sf_out, int32_t rows, int32_t KB,
+                 int32_t mma_layout, const float* __restrict__ g_seg, SegTable segs, float* __restrict__ g_shared) {
+    float gstar = 0.0f;
+    for (int j = 0; j < segs.nseg; ++j) gstar = fmaxf(gstar, __ldg(g_seg + j));
+    if (blockIdx.x == 0 && threadIdx.x == 0) *g_shared = gstar;
+    const int32_t words_per_row = (KB + 3) >> 2;
+    const int64_t total = static_cast<int64_t>(rows) * words_per_row;
+    for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < total;
+         i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        const int32_t r = static_cast<int32_t>(i / words_per_row);
+        const int32_t wq = static_cast<int32_t>(i - static_cast<int64_t>(r) * words_per_row);
+        const float ratio = __fdiv_rn(__ldg(g_seg + seg_of(segs, r)), gstar);
+        if (mma_layout) {
+            const int64_t off = sf_mma_offset(r, wq * 4, words_per_row);
+            const uint32_t w = *reinterpret_cast<const uint32_t*>(sf_in + off);
+            uint32_t o = 0;
+#pragma unroll
+            for (int b = 0; b < 4; ++b)
+                o |= f32_to_e4m3(__fmul_rn(e4m3_to_f32((w >> (8 * b)) & 0xFFu), ratio)) << (8 * b);
+            *reinterpret_cast<uint32_t*>(sf_out + off) = o;
+        } else {
+            for (int b = 0; b < 4 && wq * 4 + b < KB; ++b) {
+                const int64_t off = static_cast<int64_t>(r) * KB + wq * 4 + b;
+                sf_out[off] = static_cast<uint8_t>(f32_to_e4m3(__fmul_rn(e4m3_to_f32(sf_in[off]), ratio)));
+            }
+        }
+    }
+}
+
 // ------------------------------------------------------------------ calibration
 // max |x| as the bit pattern of a non-negative float (ordering of such patterns as
 // unsigned integers equals their ordering as floats), accumulated with atomicMax.
