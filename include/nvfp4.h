@@ -70,6 +70,10 @@ typedef enum { NVFP4_SF_LINEAR = 0, NVFP4_SF_MMA = 1 } nvfp4_sf_layout;
 /* flags for nvfp4_linear* */
 #define NVFP4_OUT_BF16 0u     /* Y is bf16 (default)                                  */
 #define NVFP4_OUT_F32  1u     /* Y is float32 (testing aid: no output rounding)       */
+#define NVFP4_WS_ZEROED 2u    /* caller's promise: the workspace was zero-filled once (e.g. cudaMemset) and has
+                                 since been written by this library only.  Lets decode-sized calls (M <= 128)
+                                 split K over several CTAs, which meet in the workspace and leave it zero again.
+                                 After NVFP4_ERR_TIMEOUT zero the workspace before the next call with this flag. */
 
 /* Size in bytes of the scale buffer for a [rows, K] tensor in `layout` (K % 16 == 0). */
 size_t nvfp4_sf_bytes(int64_t rows, int64_t K, nvfp4_sf_layout layout);
@@ -166,8 +170,10 @@ nvfp4_status nvfp4_harmonize_scales(const uint8_t* d_sf_in, int64_t N, int64_t K
  *   d_g_a              device scalar; d_g_seg device float[nseg]
  *   segs               host array (copied into the launch; need not outlive the call)
  *   d_y                out [M, N], row stride ldy elements, bf16 or float per `flags`
- *   d_workspace        nvfp4_linear_workspace_bytes(...) bytes, 16-byte aligned; its first
- *                      word is a status flag read by nvfp4_device_status
+ *   d_workspace        at least 256 bytes, 16-byte aligned; its first word is a status flag read
+ *                      by nvfp4_device_status.  nvfp4_linear_workspace_bytes(...) is the size that
+ *                      also holds the split-K area used with NVFP4_WS_ZEROED (more than 256 bytes
+ *                      only for M <= 256)
  * Requirements: K % 64 == 0; code pointers 16-byte aligned; scale pointers 16-byte aligned.
  * Errors: see nvfp4_status; M == 0 or N == 0 is a no-op.
  */
@@ -209,9 +215,10 @@ size_t nvfp4_linear_bf16_workspace_bytes(int64_t M, int64_t N, int64_t K, int ns
  * loads the library holds the array until the process exits.
  *
  *   - It calls no cudaMalloc / cudaFree and no allocating library routine.
- *   - Sizes whose nvfp4_linear_bf16_workspace_bytes(M, N, K, nseg) exceeds
- *     NVFP4_STATIC_SCRATCH_BYTES are rejected with NVFP4_ERR_WORKSPACE before anything
- *     is launched (the limit fits decode-sized batches, e.g. M = 256 rows at K = 16384).
+ *   - Sizes whose quantized activations (M*K/2 bytes of codes, their scales and a 256-byte
+ *     status block) exceed NVFP4_STATIC_SCRATCH_BYTES are rejected with NVFP4_ERR_WORKSPACE
+ *     before anything is launched (the limit fits decode-sized batches, e.g. M = 256 rows at
+ *     K = 16384).
  *   - The first call on each device looks up the array's device address (once, with that
  *     device current).  Make that first call outside of any stream capture.
  *   - All calls share the one array and it keeps the previous call's contents; the

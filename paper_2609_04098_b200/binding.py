@@ -20,6 +20,7 @@ SF_LINEAR = 0
 SF_MMA = 1
 OUT_BF16 = 0
 OUT_F32 = 1
+WS_ZEROED = 2        # workspaces from alloc_workspace are zero-filled, so the binding always promises this
 MAX_SEGMENTS = 32
 
 EXPORTS = (
@@ -232,7 +233,7 @@ def nvfp4_linear(a_codes, a_sf, g_a, w_codes, w_sf, segments, g_seg, workspace, 
     pairs = seg_pairs(segments)
     if out is None:
         out = torch.empty((M, N), dtype=torch.float32 if out_f32 else torch.bfloat16, device=a_codes.device)
-    flags = OUT_F32 if out.dtype == torch.float32 else OUT_BF16
+    flags = (OUT_F32 if out.dtype == torch.float32 else OUT_BF16) | WS_ZEROED
     _check(lib().nvfp4_linear(_ptr(a_codes), _ptr(a_sf), _ptr(g_a), M, K, _ptr(w_codes), _ptr(w_sf), N,
                               _segments(pairs), _ptr(g_seg), len(pairs), _ptr(out), out.stride(0), flags,
                               _ptr(workspace), workspace.numel(), _stream(stream)), "nvfp4_linear")
@@ -248,7 +249,7 @@ def nvfp4_linear_bf16(x, g_a, w_codes, w_sf, segments, g_seg, workspace, out=Non
     pairs = seg_pairs(segments)
     if out is None:
         out = torch.empty((M, N), dtype=torch.float32 if out_f32 else torch.bfloat16, device=x.device)
-    flags = OUT_F32 if out.dtype == torch.float32 else OUT_BF16
+    flags = (OUT_F32 if out.dtype == torch.float32 else OUT_BF16) | WS_ZEROED
     _check(lib().nvfp4_linear_bf16(_ptr(x), x.stride(0), _ptr(g_a), M, K, _ptr(w_codes), _ptr(w_sf), N,
                                    _segments(pairs), _ptr(g_seg), len(pairs), _ptr(out), out.stride(0), flags,
                                    _ptr(workspace), workspace.numel(), _stream(stream)), "nvfp4_linear_bf16")

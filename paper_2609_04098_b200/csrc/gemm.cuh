@@ -52,6 +52,13 @@ struct GemmParams {
     int32_t k_tiles;         // ceil(K / 256)
     int32_t katoms;          // K / 64: 512-byte scale atoms per 128-row band
     int32_t group_m;         // row units per raster group (see tile_of)
+    // split-K (small M): an output tile is computed by split_k CTAs, each over k_per_split
+    // consecutive K tiles; partial sums meet in `partial` (fp32 [rows padded to 128][ldp], zero
+    // between calls), `counters` (one per tile and lane quarter, zero between calls) tell the
+    // last arrival, which applies the scales, writes Y and re-zeroes what it read
+    int32_t split_k, k_per_split, ldp;
+    float* partial;
+    uint32_t* counters;
     uint32_t flags;
     uint32_t tma_store;      // 1: bf16 output through the TMA-store path (tmY valid)
     int32_t nseg;
@@ -148,9 +155,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     const uint32_t unit_id = PAIR ? (blockIdx.x >> 1) : blockIdx.x;    // CTA or cluster index
     const uint32_t n_units = PAIR ? (gridDim.x >> 1) : gridDim.x;
     const uint32_t m_units = PAIR ? (static_cast<uint32_t>(p.m_tiles) + 1u) >> 1 : static_cast<uint32_t>(p.m_tiles);
-    const uint32_t total_tiles = m_units * static_cast<uint32_t>(p.n_tiles);
+    const uint32_t split_k = static_cast<uint32_t>(p.split_k);
+    const uint32_t total_tiles = m_units * static_cast<uint32_t>(p.n_tiles) * split_k;    // work items
     const uint32_t my_tiles = total_tiles > unit_id ? (total_tiles - unit_id + n_units - 1) / n_units : 0u;
-    const uint32_t k_tiles = static_cast<uint32_t>(p.k_tiles);
+    const uint32_t k_tiles = static_cast<uint32_t>(p.k_per_split);                        // K tiles per item
     const uint32_t total_it = my_tiles * k_tiles;
     const uint32_t peer_abort =
         PAIR ? ptx::mapa_shared(ptx::smem_u32(const_cast<uint32_t*>(abort_flag)), rank ^ 1u) : 0u;
@@ -183,8 +191,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     // by the host to a fraction of L2) stay resident while the group sweeps all of W.
     const uint32_t group_m = static_cast<uint32_t>(p.group_m);
     const uint32_t tiles_per_group = group_m * static_cast<uint32_t>(p.n_tiles);
-    auto tile_of = [&](uint32_t t, int32_t& um, int32_t& un) {
-        const uint32_t tile = unit_id + t * n_units;
+    auto tile_of = [&](uint32_t t, int32_t& um, int32_t& un, int32_t& ks) {
+        const uint32_t item = unit_id + t * n_units;
+        const uint32_t tile = item / split_k;
+        ks = static_cast<int32_t>(item - tile * split_k);
         const uint32_t group = tile / tiles_per_group, r = tile - group * tiles_per_group;
         const uint32_t first = group * group_m;
         const uint32_t gsize = min(group_m, m_units - first);
@@ -211,12 +221,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             uint32_t it = 0;
             bool ok = true;
             for (uint32_t t = 0; ok && t < my_tiles; ++t) {
-                int32_t um, un;
-                tile_of(t, um, un);
+                int32_t um, un, ks;
+                tile_of(t, um, un, ks);
                 const int32_t a_band = PAIR ? 2 * um + static_cast<int32_t>(rank) : um;
                 const int32_t code_row = is_a ? a_band * kBM : un * BN + static_cast<int32_t>(rank) * C::B_ROWS;
                 const int32_t sf_band = is_a ? a_band : un * C::NB_BANDS;
-                for (int32_t kt = 0; kt < p.k_tiles; ++kt, ++it) {
+                const int32_t kt_end = (ks + 1) * p.k_per_split;        // K tiles past the tensor load zeros
+                for (int32_t kt = ks * p.k_per_split; kt < kt_end; ++kt, ++it) {
                     const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
                     if (!ptx::mbar_wait_bounded(&empty[s], ph ^ 1u, abort_flag, p.wait_limit_ns, peer_abort)) { ok = false; break; }
                     if (is_a) NVFP4_TRACE(p, 0, it);
@@ -362,8 +373,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         if (use_tma && lane == 0) ptx::prefetch_tensormap(&tmY);
         uint32_t pieces_stored = 0;
         for (uint32_t t = 0; t < my_tiles; ++t) {
-            int32_t um, un;
-            tile_of(t, um, un);
+            int32_t um, un, ks;
+            tile_of(t, um, un, ks);
             const int32_t n0 = un * BN;
             const uint32_t acc = t & 1u, aph = (t >> 1) & 1u;
             if (warp == 0 && lane == 0) NVFP4_TRACE(p, 7, t);
@@ -391,6 +402,94 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * C::ACC_STRIDE;
             const int32_t row0 = (PAIR ? 2 * um + static_cast<int32_t>(rank) : um) * kBM + quarter * 32;
             constexpr int NP = BN / kOutPieceCols;
+            if (split_k > 1u) {
+                // ---- split-K: add this item's partial sums to the tile's fp32 buffer; the last of
+                // the split_k arrivals (per lane quarter) finishes the tile
+                const int32_t row = row0 + lane;
+                const bool row_ok = row < p.M;
+                float* prow = p.partial + static_cast<int64_t>(row) * p.ldp + n0;
+#pragma unroll 1
+                for (int pc = 0; pc < NP; ++pc) {
+                    uint32_t r[64];
+                    __syncwarp();
+                    ptx::tmem_ld_32x64(t_row + pc * kOutPieceCols, r);
+                    ptx::tmem_ld_wait();
+                    if (row_ok && n0 + pc * kOutPieceCols < p.N) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            ptx::red_add_v4_f32(prow + pc * kOutPieceCols + 4 * j, __uint_as_float(r[4 * j]),
+                                                __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]),
+                                                __uint_as_float(r[4 * j + 3]));
+                    }
+                }
+                ptx::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    if (PAIR) ptx::mbar_arrive_cluster(leader_tempty + acc * 8u);
+                    else      ptx::mbar_arrive(&tempty[acc]);
+                }
+                __threadfence();                                   // my adds are visible before my ticket
+                uint32_t ticket = 0;
+                uint32_t* counter = p.counters + (static_cast<uint32_t>(um) * p.n_tiles + un) * 4u + quarter;
+                if (lane == 0) ticket = atomicAdd(counter, 1u);
+                ticket = __shfl_sync(0xffffffffu, ticket, 0);
+                if (ticket != split_k - 1u) continue;              // somebody else finishes this quarter
+                __threadfence();                                   // their adds are visible before my reads
+#pragma unroll 1
+                for (int pc = 0; pc < NP; ++pc) {
+                    const int32_t col0 = n0 + pc * kOutPieceCols;
+                    if (col0 >= p.N) break;
+                    float v[64];
+                    if (row_ok) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            float4* q4 = reinterpret_cast<float4*>(prow + pc * kOutPieceCols + 4 * j);
+                            const float4 q = __ldcg(q4);
+                            __stcg(q4, make_float4(0.0f, 0.0f, 0.0f, 0.0f));       // leave the buffer zero for the next call
+                            v[4 * j] = q.x; v[4 * j + 1] = q.y; v[4 * j + 2] = q.z; v[4 * j + 3] = q.w;
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 64; ++j) v[j] = 0.0f;
+                    }
+#pragma unroll
+                    for (int j = 0; j < 64; ++j)
+                        v[j] = __fmul_rn(v[j], __shfl_sync(0xffffffffu, areg[pc * 2 + (j >> 5)], j & 31));
+                    if (!row_ok) continue;
+                    const bool vec_ok = (reinterpret_cast<uintptr_t>(p.y) & 15u) == 0 && (p.ldy & (out_f32 ? 3 : 7)) == 0 &&
+                                        col0 + kOutPieceCols <= p.N;
+                    if (out_f32) {
+                        float* yr = reinterpret_cast<float*>(p.y) + static_cast<int64_t>(row) * p.ldy + col0;
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            if (vec_ok) {
+                                *reinterpret_cast<float4*>(yr + 4 * j) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                            } else {
+#pragma unroll
+                                for (int e = 0; e < 4; ++e)
+                                    if (col0 + 4 * j + e < p.N) yr[4 * j + e] = v[4 * j + e];
+                            }
+                        }
+                    } else {
+                        __nv_bfloat16* yr = reinterpret_cast<__nv_bfloat16*>(p.y) + static_cast<int64_t>(row) * p.ldy + col0;
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            if (vec_ok) {
+                                *reinterpret_cast<uint4*>(yr + 8 * j) =
+                                    make_uint4(pack_bf16x2(v[8 * j], v[8 * j + 1]), pack_bf16x2(v[8 * j + 2], v[8 * j + 3]),
+                                               pack_bf16x2(v[8 * j + 4], v[8 * j + 5]), pack_bf16x2(v[8 * j + 6], v[8 * j + 7]));
+                            } else {
+#pragma unroll
+                                for (int e = 0; e < 8; ++e)
+                                    if (col0 + 8 * j + e < p.N) yr[8 * j + e] = __float2bfloat16_rn(v[8 * j + e]);
+                            }
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) *counter = 0u;                      // ready for the next call
+                continue;
+            }
             // piece order: with overlapping accumulators the shared columns go first (the last piece
             // of the lower accumulator, the first piece of the upper one)
             auto drain = [&](auto first_c) {

@@ -199,7 +199,7 @@ nvfp4_status launch_gemm(const GemmMaps& tm, GemmParams& p, int sm_count, cudaSt
     cudaGetDevice(&dev);
     p.n_tiles = (p.N + BN - 1) / BN;
     const int64_t m_units = PAIR ? (p.m_tiles + 1) / 2 : p.m_tiles;
-    const int64_t tiles = m_units * p.n_tiles;
+    const int64_t tiles = m_units * p.n_tiles * (p.split_k > 0 ? p.split_k : 1);
     {
         // rows of A kept live per raster group: about 32 MB of codes and scales (a quarter of L2)
         const int64_t unit_bytes = static_cast<int64_t>(PAIR ? 256 : 128) * (p.K / 2 + p.K / 16);
@@ -253,6 +253,7 @@ int choose_variant(int64_t M, int64_t N) {
     const int forced = g_variant.load(std::memory_order_relaxed);
     if (forced != 0) return forced;
     if (M > 128 && N >= 256) return 2;
+    if (M <= 128) return 128;                 // decode-sized: more, smaller tiles (and split-K)
     return N >= 256 ? 256 : 128;
 }
 
@@ -327,6 +328,23 @@ nvfp4_status check_quantize_args(const void* d_x, int64_t rows, int64_t K, int64
 }
 
 constexpr size_t kStatusBytes = 256;
+
+// split-K area of a workspace (after the status block): counters, then fp32 partial sums
+struct SplitArea {
+    size_t counters_bytes = 0, partial_bytes = 0;
+    int64_t ldp = 0;
+    size_t total() const { return counters_bytes + partial_bytes; }
+};
+SplitArea split_area(int64_t M, int64_t N) {
+    SplitArea a;
+    if (M <= 0 || N <= 0 || M > 256) return a;                 // split-K serves decode-sized batches only
+    const int64_t m_tiles = (M + 127) / 128, n_tiles = (N + 127) / 128;
+    a.counters_bytes = (static_cast<size_t>(m_tiles * n_tiles * 4) * sizeof(uint32_t) + 255) & ~static_cast<size_t>(255);
+    a.ldp = n_tiles * 128;
+    a.partial_bytes = static_cast<size_t>(m_tiles * 128) * static_cast<size_t>(a.ldp) * sizeof(float);
+    if (a.partial_bytes > (64u << 20)) return SplitArea();
+    return a;
+}
 
 }  // namespace
 }  // namespace nvfp4
@@ -460,7 +478,10 @@ nvfp4_status nvfp4_harmonize_scales(const uint8_t* d_sf_in, int64_t N, int64_t K
     return cudaGetLastError() == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
 
-size_t nvfp4_linear_workspace_bytes(int64_t, int64_t, int64_t, int) { return kStatusBytes; }
+size_t nvfp4_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int nseg) {
+    (void)K; (void)nseg;
+    return kStatusBytes + split_area(M, N).total();
+}
 
 nvfp4_status nvfp4_workspace_reset(void* d_workspace, size_t workspace_bytes, void* stream) {
     if (d_workspace == nullptr) return NVFP4_ERR_NULL;
@@ -468,10 +489,15 @@ nvfp4_status nvfp4_workspace_reset(void* d_workspace, size_t workspace_bytes, vo
     return cudaMemsetAsync(d_workspace, 0, kStatusBytes, as_stream(stream)) == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
 
-nvfp4_status nvfp4_linear(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const float* d_g_a, int64_t M,
-                          int64_t K, const uint8_t* d_w_codes, const uint8_t* d_w_sf, int64_t N,
-                          const nvfp4_segment* segs, const float* d_g_seg, int nseg, void* d_y, int64_t ldy,
-                          uint32_t flags, void* d_workspace, size_t workspace_bytes, void* stream) {
+}  // extern "C"
+
+namespace {
+// `d_split` / `split_bytes`: zero-filled split-K area (may be null: then no split-K)
+nvfp4_status linear_impl(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const float* d_g_a, int64_t M,
+                         int64_t K, const uint8_t* d_w_codes, const uint8_t* d_w_sf, int64_t N,
+                         const nvfp4_segment* segs, const float* d_g_seg, int nseg, void* d_y, int64_t ldy,
+                         uint32_t flags, void* d_workspace, size_t workspace_bytes, void* d_split, size_t split_bytes,
+                         void* stream, int64_t a_rows_alloc = 0) {
     if (d_a_codes == nullptr || d_a_sf == nullptr || d_g_a == nullptr || d_w_codes == nullptr ||
         d_w_sf == nullptr || d_g_seg == nullptr || d_y == nullptr)
         return NVFP4_ERR_NULL;
@@ -484,7 +510,7 @@ nvfp4_status nvfp4_linear(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const
         return NVFP4_ERR_ALIGN;
     if (d_workspace == nullptr || workspace_bytes < kStatusBytes) return NVFP4_ERR_WORKSPACE;
     if (!aligned16(d_workspace)) return NVFP4_ERR_ALIGN;
-    if ((flags & ~NVFP4_OUT_F32) != 0u) return NVFP4_ERR_SHAPE;
+    if ((flags & ~(NVFP4_OUT_F32 | NVFP4_WS_ZEROED)) != 0u) return NVFP4_ERR_SHAPE;
     if (M == 0 || N == 0) return NVFP4_OK;
     DeviceInfo info;
     st = check_arch(info);
@@ -494,7 +520,9 @@ nvfp4_status nvfp4_linear(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const
     const int tile_n = bn == 128 ? 128 : 256;
     GemmMaps tm;
     std::memset(&tm, 0, sizeof(tm));
-    st = codes_tensor_map(d_a_codes, M, K, kBM, &tm.a);
+    // rows the code buffer really has (>= M): with whole 128-row boxes in bounds TMA takes no
+    // out-of-bounds path, which is measurably slower; rows past M hold zero scales and are never stored
+    st = codes_tensor_map(d_a_codes, a_rows_alloc > M ? a_rows_alloc : M, K, kBM, &tm.a);
     if (st != NVFP4_OK) return st;
     st = codes_tensor_map(d_w_codes, N, K, bn == 2 ? 128 : tile_n, &tm.b);
     if (st != NVFP4_OK) return st;
@@ -521,6 +549,23 @@ nvfp4_status nvfp4_linear(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const
     p.m_tiles = static_cast<int32_t>((M + kBM - 1) / kBM);
     p.k_tiles = static_cast<int32_t>((K + 255) / 256);
     p.katoms = static_cast<int32_t>(K / 64);
+    p.split_k = 1;
+    p.k_per_split = p.k_tiles;
+    if (bn == 128 && (flags & NVFP4_WS_ZEROED) != 0u && d_split != nullptr && (K % 256) == 0) {
+        // small M: too few tiles for the machine -> several CTAs share a tile along K
+        const SplitArea area = split_area(M, N);
+        const int64_t tiles = static_cast<int64_t>(p.m_tiles) * ((N + 127) / 128);
+        int64_t want = tiles > 0 ? info.sm_count / tiles : 1;
+        if (want > p.k_tiles) want = p.k_tiles;
+        // pays only when the K loop is long: the meeting in the workspace costs about 4 us of latency
+        if (area.total() > 0 && split_bytes >= area.total() && want >= 2 && p.k_tiles >= 32) {
+            p.k_per_split = static_cast<int32_t>((p.k_tiles + want - 1) / want);
+            p.split_k = static_cast<int32_t>((p.k_tiles + p.k_per_split - 1) / p.k_per_split);
+            p.counters = reinterpret_cast<uint32_t*>(d_split);
+            p.partial = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(d_split) + area.counters_bytes);
+            p.ldp = static_cast<int32_t>(area.ldp);
+        }
+    }
     p.flags = flags;
     p.nseg = nseg;
     for (int i = 0; i < nseg; ++i) p.seg_end[i] = static_cast<int32_t>(segs[i].col_begin + segs[i].col_count);
@@ -541,11 +586,37 @@ nvfp4_status nvfp4_linear(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const
     }
 }
 
+// workspace of the fused call: [status][codes][scales][optional split-K area]
+size_t fused_codes_bytes(int64_t M, int64_t K) {        // rows padded to whole 128-row tiles
+    const int64_t m_pad = (M + 127) / 128 * 128;
+    return (static_cast<size_t>(m_pad) * static_cast<size_t>(K / 2) + 255) & ~static_cast<size_t>(255);
+}
+size_t fused_min_bytes(int64_t M, int64_t K) {
+    const size_t sf = (nvfp4_sf_bytes(M, K, NVFP4_SF_MMA) + 255) & ~static_cast<size_t>(255);
+    return kStatusBytes + fused_codes_bytes(M, K) + sf;
+}
+}  // namespace
+
+extern "C" {
+
+nvfp4_status nvfp4_linear(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const float* d_g_a, int64_t M,
+                          int64_t K, const uint8_t* d_w_codes, const uint8_t* d_w_sf, int64_t N,
+                          const nvfp4_segment* segs, const float* d_g_seg, int nseg, void* d_y, int64_t ldy,
+                          uint32_t flags, void* d_workspace, size_t workspace_bytes, void* stream) {
+    void* split = nullptr;
+    size_t split_bytes = 0;
+    if (d_workspace != nullptr && workspace_bytes > kStatusBytes) {
+        split = reinterpret_cast<uint8_t*>(d_workspace) + kStatusBytes;
+        split_bytes = workspace_bytes - kStatusBytes;
+    }
+    return linear_impl(d_a_codes, d_a_sf, d_g_a, M, K, d_w_codes, d_w_sf, N, segs, d_g_seg, nseg, d_y, ldy, flags,
+                       d_workspace, workspace_bytes, split, split_bytes, stream);
+}
+
 size_t nvfp4_linear_bf16_workspace_bytes(int64_t M, int64_t N, int64_t K, int nseg) {
-    (void)N; (void)nseg;
+    (void)nseg;
     if (M < 0 || K < 0 || (K % 16) != 0) return 0;
-    const size_t codes = (static_cast<size_t>(M) * static_cast<size_t>(K / 2) + 255) & ~static_cast<size_t>(255);
-    return kStatusBytes + codes + nvfp4_sf_bytes(M, K, NVFP4_SF_MMA);
+    return fused_min_bytes(M, K) + split_area(M, N).total();
 }
 
 nvfp4_status nvfp4_linear_bf16(const void* d_x, int64_t ldx, const float* d_g_a, int64_t M, int64_t K,
@@ -554,16 +625,16 @@ nvfp4_status nvfp4_linear_bf16(const void* d_x, int64_t ldx, const float* d_g_a,
                                uint32_t flags, void* d_workspace, size_t workspace_bytes, void* stream) {
     if (d_workspace == nullptr) return NVFP4_ERR_WORKSPACE;
     if (M < 0 || K <= 0 || (K % 64) != 0) return NVFP4_ERR_SHAPE;
-    if (workspace_bytes < nvfp4_linear_bf16_workspace_bytes(M, N, K, nseg)) return NVFP4_ERR_WORKSPACE;
+    const size_t min_bytes = fused_min_bytes(M, K);
+    if (workspace_bytes < min_bytes) return NVFP4_ERR_WORKSPACE;
     if (!aligned16(d_workspace)) return NVFP4_ERR_ALIGN;
     uint8_t* ws = reinterpret_cast<uint8_t*>(d_workspace);
     uint8_t* codes = ws + kStatusBytes;
-    const size_t codes_bytes = (static_cast<size_t>(M) * static_cast<size_t>(K / 2) + 255) & ~static_cast<size_t>(255);
-    uint8_t* sf = codes + codes_bytes;
+    uint8_t* sf = codes + fused_codes_bytes(M, K);
     nvfp4_status st = nvfp4_quantize_act(d_x, M, K, ldx, d_g_a, codes, sf, NVFP4_SF_MMA, stream);
     if (st != NVFP4_OK) return st;
-    return nvfp4_linear(codes, sf, d_g_a, M, K, d_w_codes, d_w_sf, N, segs, d_g_seg, nseg, d_y, ldy, flags,
-                        d_workspace, kStatusBytes, stream);
+    return linear_impl(codes, sf, d_g_a, M, K, d_w_codes, d_w_sf, N, segs, d_g_seg, nseg, d_y, ldy, flags, d_workspace,
+                       kStatusBytes, ws + min_bytes, workspace_bytes - min_bytes, stream, (M + 127) / 128 * 128);
 }
 
 // ---------------------------------------------------------------- no-allocation variant
@@ -596,15 +667,18 @@ nvfp4_status nvfp4_linear_bf16_static(const void* d_x, int64_t ldx, const float*
                                       const nvfp4_segment* segs, const float* d_g_seg, int nseg, void* d_y,
                                       int64_t ldy, uint32_t flags, void* stream) {
     if (M < 0 || K <= 0 || (K % 64) != 0) return NVFP4_ERR_SHAPE;
-    const size_t need = nvfp4_linear_bf16_workspace_bytes(M, N, K, nseg);
+    (void)N;
+    const size_t need = (K % 16) == 0 ? fused_min_bytes(M, K) : 0;
     if (need == 0 || need > NVFP4_STATIC_SCRATCH_BYTES) return NVFP4_ERR_WORKSPACE;   // beyond the fixed array
     void* scratch = nullptr;
     nvfp4_status st = static_scratch_address(&scratch);
     if (st != NVFP4_OK) return st;
     st = nvfp4_workspace_reset(scratch, NVFP4_STATIC_SCRATCH_BYTES, stream);           // status word starts at zero
     if (st != NVFP4_OK) return st;
-    return nvfp4_linear_bf16(d_x, ldx, d_g_a, M, K, d_w_codes, d_w_sf, N, segs, d_g_seg, nseg, d_y, ldy, flags,
-                             scratch, NVFP4_STATIC_SCRATCH_BYTES, stream);
+    // the array starts as zeros (static storage) and only this library writes it, leaving its
+    // split-K part zero after every call: the NVFP4_WS_ZEROED promise holds by construction
+    return nvfp4_linear_bf16(d_x, ldx, d_g_a, M, K, d_w_codes, d_w_sf, N, segs, d_g_seg, nseg, d_y, ldy,
+                             flags | NVFP4_WS_ZEROED, scratch, NVFP4_STATIC_SCRATCH_BYTES, stream);
 }
 
 nvfp4_status nvfp4_static_status(void* stream) {

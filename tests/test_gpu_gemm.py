@@ -220,3 +220,29 @@ def test_gdn_in_projection_full_size_sampled(variant):
     scale = np.linalg.norm(a_hat, axis=1) * np.linalg.norm(w_hat) / np.sqrt(K)
     # bf16 rounding of N outputs: random-walk error ~ 2^-9 * |y| * sqrt(N)
     assert np.max(np.abs(got - want) / scale) < 2e-2
+
+
+# ---- decode-sized batches: split-K over a self-cleaning workspace -----------------------------
+@pytest.mark.parametrize("M,N,K", [(1, 6144, 5120), (16, 520, 8192), (100, 2064, 8448), (128, 1000, 9216), (3, 136, 17408)])
+@pytest.mark.parametrize("out_f32", [False, True])
+def test_small_m_split_k(M, N, K, out_f32):
+    n1 = N // 3
+    segs, x, w, ac, asf, ga, wc, wsf, gs = _oracle_operands(17, M, K, (("p", n1, 0.02), ("q", N - n1, 0.2)))
+    gcol = oracle.col_scales(N, segs, gs)
+    y_ref = oracle.gemm(ac, asf, ga, wc, wsf, gcol)
+    bound = gu.gemm_bounds(ac, asf, ga, wc, wsf, gcol)
+    ws = nv.alloc_workspace(gu.DEV, M, N, K, 2)            # zero-filled, large enough for the split-K area
+    assert ws.numel() > 256
+    first = None
+    for _ in range(3):                                      # the same workspace every time: it must come back clean
+        y = _run_from_oracle_operands(segs, ac, asf, ga, wc, wsf, gs, K, out_f32=out_f32, ws=ws)
+        gu.check_gemm(y, y_ref, bound, "split-K %s" % ((M, N, K),))
+        if first is None:
+            first = y.clone()
+        elif out_f32:
+            # fp32 atomics add in arrival order: equal up to summation order
+            assert torch.allclose(y, first, rtol=1e-5, atol=1e-6 * float(first.abs().max()))
+    assert bool((ws[256:] == 0).all())                     # counters and partial sums left at zero
+    # and the one-tile-per-CTA kernel gives the same answer (within summation order)
+    y1 = _run_from_oracle_operands(segs, ac, asf, ga, wc, wsf, gs, K, out_f32=out_f32)    # 256-byte workspace: no split
+    gu.check_gemm(y1, y_ref, bound, "no split")
