@@ -55,13 +55,6 @@ __device__ __forceinline__ uint32_t f32x8_to_e2m1(const float (&y)[8]) {
     return out;
 }
 
-__device__ __forceinline__ void bf16x8_to_f32(const uint4& v, float (&f)[8]) {
-    f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xFFFF0000u);
-    f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xFFFF0000u);
-    f[4] = __uint_as_float(v.z << 16); f[5] = __uint_as_float(v.z & 0xFFFF0000u);
-    f[6] = __uint_as_float(v.w << 16); f[7] = __uint_as_float(v.w & 0xFFFF0000u);
-}
-
 // Byte offset of scale (row r, block b) in the tensor-core layout; katoms = ceil(K/64).
 __device__ __forceinline__ int64_t sf_mma_offset(int32_t r, int32_t b, int32_t katoms) {
     const int32_t rr = r & 127;
