@@ -412,6 +412,18 @@ def run_gpu(args):
         c1.record(stream)
         torch.cuda.synchronize()
         cal_ms = c0.elapsed_time(c1) / reps
+        # the same tensor through the RMSNorm-fused quantizer (norm gain ~ 1)
+        wn = torch.ones(HIDDEN, dtype=torch.bfloat16, device=dev)
+        for i in range(nbuf):
+            nv.nvfp4_rmsnorm_quantize(xq[i % nbuf], wn, 1e-6, gq, out=outs[i % nbuf])
+        torch.cuda.synchronize()
+        n0, n1 = ev(), ev()
+        n0.record(stream)
+        for i in range(reps):
+            nv.nvfp4_rmsnorm_quantize(xq[i % nbuf], wn, 1e-6, gq, out=outs[i % nbuf])
+        n1.record(stream)
+        torch.cuda.synchronize()
+        rms_ms = n0.elapsed_time(n1) / reps
         result["quantize"] = {
             "workload": "configs[1] activation quantize 8192x5120 bf16, heavy-tailed; %d rotating buffers" % nbuf,
             "metric": "act_quantize_gbs", "value": round(q_gbs, 1), "unit": "GB/s", "us_per_call": round(q_ms * 1e3, 2),
@@ -421,6 +433,8 @@ def run_gpu(args):
                          "frac_of_nominal_8tbs": round(q_gbs / NOMINAL_HBM_GBS, 4),
                          "traffic": ncu_traffic("quantize_kernel")},
             "calibrate_gbs": round(8192 * HIDDEN * 2 / (cal_ms * 1e-3) / 1e9, 1),
+            "rmsnorm_quantize": {"us_per_call": round(rms_ms * 1e3, 2), "value": round(q_bytes / (rms_ms * 1e-3) / 1e9, 1),
+                                 "unit": "GB/s", "note": "RMSNorm fused in front: same HBM bytes, row read twice (second time from cache)"},
             "in_step_gbs": None if quant_in_step_gbs is None else round(quant_in_step_gbs, 1)}
         del xq, outs
 

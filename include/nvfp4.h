@@ -126,6 +126,23 @@ nvfp4_status nvfp4_swiglu_quantize(const void* d_gate_up, int64_t M, int64_t inn
                                    nvfp4_sf_layout layout, void* stream);
 
 /*
+ * Activation quantization fused into RMSNorm (paper: Background / Setup -- norms are excluded from
+ * quantization and stay bf16 upstream of every quantized linear, so the in-projections quantize
+ * a normalised residual stream on every call).  One pass over x from HBM:
+ *     y = bf16_rne( (x * rstd) * w ),  rstd = 1 / sqrt(mean_k(x^2) + eps),  then nvfp4_quantize_act(y)
+ * in binary32: each of 32 lanes sums x^2 (fused multiply-add) over the 16-element pieces k/16 % 32
+ * == lane in increasing k, the partial sums meet in a butterfly (offsets 16, 8, 4, 2, 1), IEEE
+ * divide, sqrt and reciprocal.
+ *   d_x       bf16 [M, K], row stride ld; 32-byte aligned, ld % 16 == 0
+ *   d_weight  bf16 [K] (the norm's gain), 32-byte aligned;  eps >= 0
+ *   d_g       in: global scale of y (calibrated offline);  outputs as nvfp4_quantize_act
+ * Errors: as nvfp4_quantize_act, plus NULL / misaligned weight, negative or NaN eps.
+ */
+nvfp4_status nvfp4_rmsnorm_quantize(const void* d_x, int64_t M, int64_t K, int64_t ld, const void* d_weight,
+                                    float eps, const float* d_g, uint8_t* d_codes, uint8_t* d_sf,
+                                    nvfp4_sf_layout layout, void* stream);
+
+/*
  * Offline weight quantization, same format, blocks along K, with one global scale
  * per fused module (paper: Section 6 -- the calibration tool keeps one FP32 global
  * scale per linear module; the modules are later served as one fused GEMM).

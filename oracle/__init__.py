@@ -66,6 +66,8 @@ def _load():
     L.orc_silu_mul.argtypes = [ctypes.c_float, ctypes.c_float]
     L.orc_swiglu_bf16.restype = None
     L.orc_swiglu_bf16.argtypes = [u16p, i64, i64, i64, u16p]
+    L.orc_rmsnorm_bf16.restype = None
+    L.orc_rmsnorm_bf16.argtypes = [u16p, i64, i64, i64, u16p, ctypes.c_float, u16p]
     L.orc_dequantize.restype = None
     L.orc_dequantize.argtypes = [u8p, u8p, f32p, i64, i64, f64p]
     L.orc_harmonize_scales.restype = ctypes.c_float
@@ -177,6 +179,17 @@ def swiglu_bf16(gate_up_bits: np.ndarray) -> np.ndarray:
     h = np.empty((R, two_i // 2), np.uint16)
     _load().orc_swiglu_bf16(_p(gu), R, two_i // 2, two_i, _p(h))
     return h
+
+
+def rmsnorm_bf16(x_bits: np.ndarray, w_bits: np.ndarray, eps: float) -> np.ndarray:
+    """bf16 [R, C], weight bf16 [C] -> bf16( x / sqrt(mean(x^2) + eps) * w ), bit patterns [R, C]."""
+    x = _c(x_bits, np.uint16)
+    w = _c(w_bits, np.uint16)
+    R, C = x.shape
+    assert w.shape == (C,)
+    y = np.empty((R, C), np.uint16)
+    _load().orc_rmsnorm_bf16(_p(x), R, C, C, _p(w), ctypes.c_float(float(np.float32(eps))), _p(y))
+    return y
 
 
 def dequantize(codes: np.ndarray, sf: np.ndarray, g_row: np.ndarray) -> np.ndarray:

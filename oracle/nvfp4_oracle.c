@@ -227,6 +227,40 @@ void orc_swiglu_bf16(const uint16_t* gate_up, int64_t rows, int64_t inner, int64
                                                             bf16_to_f32(gate_up[r * ld + inner + c])));
 }
 
+/* ------------------------------------------------------------------------- */
+/* Producer fusion for the in-projections: their input is RMSNorm(x) * w (the  */
+/* norms stay bf16 upstream of every quantized linear).  The paper fixes no    */
+/* arithmetic for it; the contract is this binary32 sequence (fmaf fused):     */
+/*   the row is dealt to 32 lanes in 16-element pieces (element k belongs to   */
+/*   lane (k/16) % 32); each lane accumulates ss = fmaf(x, x, ss) over its     */
+/*   elements in increasing k; the 32 partial sums meet in a butterfly         */
+/*   (ss[l] += ss[l ^ off], off = 16, 8, 4, 2, 1);                             */
+/*   rstd = 1 / sqrt(ss / K + eps);   y = bf16_rne( (x * rstd) * w )           */
+/* ------------------------------------------------------------------------- */
+void orc_rmsnorm_bf16(const uint16_t* x, int64_t rows, int64_t cols, int64_t ld, const uint16_t* w, float eps,
+                      uint16_t* y) {
+    #pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r) {
+        float ss[32], t[32];
+        for (int l = 0; l < 32; ++l) ss[l] = 0.0f;
+        for (int64_t k = 0; k < cols; ++k) {
+            const float v = bf16_to_f32(x[r * ld + k]);
+            const int l = (int)((k / 16) % 32);
+            ss[l] = fmaf(v, v, ss[l]);
+        }
+        for (int off = 16; off >= 1; off >>= 1) {
+            for (int l = 0; l < 32; ++l) t[l] = ss[l] + ss[l ^ off];
+            for (int l = 0; l < 32; ++l) ss[l] = t[l];
+        }
+        const float mean = ss[0] / (float)cols;
+        const float rstd = 1.0f / sqrtf(mean + eps);
+        for (int64_t k = 0; k < cols; ++k) {
+            const float v = bf16_to_f32(x[r * ld + k]) * rstd;
+            y[r * cols + k] = orc_f32_to_bf16(v * bf16_to_f32(w[k]));
+        }
+    }
+}
+
 /* x_hat = e2m1(code) * e4m3(scale) * g, evaluated in double (every factor is a
  * binary32 with few significant bits, so the double product is exact). */
 void orc_dequantize(const uint8_t* codes, const uint8_t* sf, const float* g_row,

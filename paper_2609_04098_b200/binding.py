@@ -24,7 +24,8 @@ WS_ZEROED = 2        # workspaces from alloc_workspace are zero-filled, so the b
 MAX_SEGMENTS = 32
 
 EXPORTS = (
-    "nvfp4_sf_bytes", "nvfp4_calibrate", "nvfp4_quantize_act", "nvfp4_swiglu_quantize", "nvfp4_quantize_weight",
+    "nvfp4_sf_bytes", "nvfp4_calibrate", "nvfp4_quantize_act", "nvfp4_swiglu_quantize", "nvfp4_rmsnorm_quantize",
+    "nvfp4_quantize_weight",
     "nvfp4_harmonize_scales", "nvfp4_linear", "nvfp4_linear_workspace_bytes", "nvfp4_linear_bf16",
     "nvfp4_linear_bf16_workspace_bytes", "nvfp4_linear_bf16_static", "nvfp4_static_status", "nvfp4_workspace_reset", "nvfp4_device_status",
     "nvfp4_set_wait_limit_ns", "nvfp4_selftest_bounded_wait", "nvfp4_launch_count", "nvfp4_set_gemm_variant", "nvfp4_gemm_variants", "nvfp4_status_string",
@@ -62,6 +63,8 @@ def lib() -> ctypes.CDLL:
     L.nvfp4_quantize_act.argtypes = [vp, i64, i64, i64, vp, vp, vp, i32, vp]
     L.nvfp4_swiglu_quantize.restype = i32
     L.nvfp4_swiglu_quantize.argtypes = [vp, i64, i64, i64, vp, vp, vp, i32, vp]
+    L.nvfp4_rmsnorm_quantize.restype = i32
+    L.nvfp4_rmsnorm_quantize.argtypes = [vp, i64, i64, i64, vp, ctypes.c_float, vp, vp, vp, i32, vp]
     L.nvfp4_quantize_weight.restype = i32
     L.nvfp4_quantize_weight.argtypes = [vp, i64, i64, i64, segp, i32, vp, i32, vp, vp, i32, vp]
     L.nvfp4_harmonize_scales.restype = i32
@@ -186,6 +189,18 @@ def nvfp4_swiglu_quantize(gate_up: torch.Tensor, g: torch.Tensor, layout: int = 
     codes, sf = out if out is not None else alloc_quantized(M, inner, gate_up.device, layout)
     _check(lib().nvfp4_swiglu_quantize(_ptr(gate_up), M, inner, gate_up.stride(0), _ptr(g), _ptr(codes), _ptr(sf),
                                        layout, _stream(stream)), "nvfp4_swiglu_quantize")
+    return codes, sf
+
+
+def nvfp4_rmsnorm_quantize(x: torch.Tensor, weight: torch.Tensor, eps: float, g: torch.Tensor, layout: int = SF_MMA,
+                           out=None, stream=None):
+    """bf16 [M, K], gain bf16 [K] -> NVFP4 of bf16(RMSNorm(x) * weight): (codes, scale bytes)."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
+    assert weight.dtype == torch.bfloat16 and weight.numel() == x.shape[1] and weight.is_contiguous()
+    M, K = x.shape
+    codes, sf = out if out is not None else alloc_quantized(M, K, x.device, layout)
+    _check(lib().nvfp4_rmsnorm_quantize(_ptr(x), M, K, x.stride(0), _ptr(weight), ctypes.c_float(eps), _ptr(g),
+                                        _ptr(codes), _ptr(sf), layout, _stream(stream)), "nvfp4_rmsnorm_quantize")
     return codes, sf
 
 

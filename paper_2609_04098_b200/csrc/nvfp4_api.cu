@@ -257,16 +257,17 @@ int choose_variant(int64_t M, int64_t N) {
     return N >= 256 ? 256 : 128;
 }
 
-template <bool MMA, bool SWIGLU>
+template <bool MMA, int MODE>
 nvfp4_status launch_quantize(const uint16_t* x, int64_t M, int64_t K, int64_t ld, const float* d_g,
                              const SegTable& segs, uint8_t* d_codes, uint8_t* d_sf, int64_t chunks, int64_t per_unit,
-                             int64_t units_per_row, int64_t units, int sm_count, cudaStream_t stream) {
+                             int64_t units_per_row, int64_t units, int sm_count, cudaStream_t stream,
+                             const uint16_t* aux, float eps) {
     constexpr int kUnroll = 2;
     // persistent grid: exactly what is resident at once, so that no partial second wave forms
     static std::atomic<int> per_sm_cache{0};
     int per_sm = per_sm_cache.load(std::memory_order_relaxed);
     if (per_sm == 0) {
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, quantize_kernel<MMA, kUnroll, SWIGLU>, 256, 0) !=
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, quantize_kernel<MMA, kUnroll, MODE>, 256, 0) !=
                 cudaSuccess || per_sm < 1) {
             cudaGetLastError();
             per_sm = 4;
@@ -277,8 +278,8 @@ nvfp4_status launch_quantize(const uint16_t* x, int64_t M, int64_t K, int64_t ld
     const int64_t max_blocks = static_cast<int64_t>(sm_count) * per_sm;
     if (blocks > max_blocks) blocks = max_blocks;
     if (blocks < 1) blocks = 1;
-    quantize_kernel<MMA, kUnroll, SWIGLU><<<static_cast<int>(blocks), 256, 0, stream>>>(
-        x, static_cast<int32_t>(M), static_cast<int32_t>(K), ld, d_g, segs, d_codes, d_sf,
+    quantize_kernel<MMA, kUnroll, MODE><<<static_cast<int>(blocks), 256, 0, stream>>>(
+        x, static_cast<int32_t>(M), static_cast<int32_t>(K), ld, d_g, segs, aux, eps, d_codes, d_sf,
         static_cast<int32_t>(chunks), static_cast<int32_t>(per_unit), static_cast<int32_t>(units_per_row),
         static_cast<int32_t>(units));
     g_launches.fetch_add(1, std::memory_order_relaxed);
@@ -287,7 +288,8 @@ nvfp4_status launch_quantize(const uint16_t* x, int64_t M, int64_t K, int64_t ld
 
 nvfp4_status quantize_impl(const void* d_x, int64_t M, int64_t K, int64_t ld, const float* d_g,
                            const SegTable& segs, uint8_t* d_codes, uint8_t* d_sf, nvfp4_sf_layout layout,
-                           const DeviceInfo& info, cudaStream_t stream, bool swiglu = false) {
+                           const DeviceInfo& info, cudaStream_t stream, int mode = kQuantPlain,
+                           const uint16_t* aux = nullptr, float eps = 0.0f) {
     const int64_t chunks = (K + 511) / 512;              // 512 elements = one block per lane
     if (M >= (1ll << 31) || K >= (1ll << 31)) return NVFP4_ERR_SHAPE;
     if (layout == NVFP4_SF_MMA && (M % 128) != 0) {
@@ -300,21 +302,20 @@ nvfp4_status quantize_impl(const void* d_x, int64_t M, int64_t K, int64_t ld, co
     // a unit = up to `per_unit` consecutive chunks of one row, handled by one warp
     constexpr int kUnroll = 2;      // matches launch_quantize
     const int64_t resident_warps = static_cast<int64_t>(info.sm_count) * 40;   // 5 blocks of 8 warps per SM
-    const int64_t per_unit = (M * chunks > 2 * resident_warps) ? kUnroll : 1;
+    int64_t per_unit = (M * chunks > 2 * resident_warps) ? kUnroll : 1;
+    if (mode == kQuantRmsnorm) per_unit = chunks;           // the row reduction needs the whole row in one warp
     const int64_t units_per_row = (chunks + per_unit - 1) / per_unit;
     const int64_t units = M * units_per_row;
     if (units >= (1ll << 31)) return NVFP4_ERR_SHAPE;
     const uint16_t* x = reinterpret_cast<const uint16_t*>(d_x);
     const bool mma = layout == NVFP4_SF_MMA;
-    if (swiglu)
-        return mma ? launch_quantize<true, true>(x, M, K, ld, d_g, segs, d_codes, d_sf, chunks, per_unit, units_per_row,
-                                                 units, info.sm_count, stream)
-                   : launch_quantize<false, true>(x, M, K, ld, d_g, segs, d_codes, d_sf, chunks, per_unit, units_per_row,
-                                                  units, info.sm_count, stream);
-    return mma ? launch_quantize<true, false>(x, M, K, ld, d_g, segs, d_codes, d_sf, chunks, per_unit, units_per_row,
-                                              units, info.sm_count, stream)
-               : launch_quantize<false, false>(x, M, K, ld, d_g, segs, d_codes, d_sf, chunks, per_unit, units_per_row,
-                                               units, info.sm_count, stream);
+#define NVFP4_LAUNCH_Q(MMA_, MODE_)                                                                          \
+    launch_quantize<MMA_, MODE_>(x, M, K, ld, d_g, segs, d_codes, d_sf, chunks, per_unit, units_per_row, units, \
+                                 info.sm_count, stream, aux, eps)
+    if (mode == kQuantSwiglu) return mma ? NVFP4_LAUNCH_Q(true, kQuantSwiglu) : NVFP4_LAUNCH_Q(false, kQuantSwiglu);
+    if (mode == kQuantRmsnorm) return mma ? NVFP4_LAUNCH_Q(true, kQuantRmsnorm) : NVFP4_LAUNCH_Q(false, kQuantRmsnorm);
+    return mma ? NVFP4_LAUNCH_Q(true, kQuantPlain) : NVFP4_LAUNCH_Q(false, kQuantPlain);
+#undef NVFP4_LAUNCH_Q
 }
 
 nvfp4_status check_quantize_args(const void* d_x, int64_t rows, int64_t K, int64_t ld, const float* d_g,
@@ -442,7 +443,7 @@ nvfp4_status nvfp4_swiglu_quantize(const void* d_gate_up, int64_t M, int64_t inn
     if (st != NVFP4_OK) return st;
     SegTable segs;
     std::memset(&segs, 0, sizeof(segs));
-    return quantize_impl(d_gate_up, M, inner, ld, d_g, segs, d_codes, d_sf, layout, info, as_stream(stream), true);
+    return quantize_impl(d_gate_up, M, inner, ld, d_g, segs, d_codes, d_sf, layout, info, as_stream(stream), kQuantSwiglu);
 }
 
 nvfp4_status nvfp4_harmonize_scales(const uint8_t* d_sf_in, int64_t N, int64_t K, nvfp4_sf_layout layout,
@@ -476,6 +477,24 @@ nvfp4_status nvfp4_harmonize_scales(const uint8_t* d_sf_in, int64_t N, int64_t K
                                                              d_g_seg, table, d_g_shared);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+}
+
+nvfp4_status nvfp4_rmsnorm_quantize(const void* d_x, int64_t M, int64_t K, int64_t ld, const void* d_weight, float eps,
+                                    const float* d_g, uint8_t* d_codes, uint8_t* d_sf, nvfp4_sf_layout layout,
+                                    void* stream) {
+    nvfp4_status st = check_quantize_args(d_x, M, K, ld, d_g, d_codes, d_sf, layout);
+    if (st != NVFP4_OK) return st;
+    if (d_weight == nullptr) return NVFP4_ERR_NULL;
+    if ((reinterpret_cast<uintptr_t>(d_weight) & 31u) != 0) return NVFP4_ERR_ALIGN;
+    if (!(eps >= 0.0f)) return NVFP4_ERR_SHAPE;
+    if (M == 0) return NVFP4_OK;
+    DeviceInfo info;
+    st = check_arch(info);
+    if (st != NVFP4_OK) return st;
+    SegTable segs;
+    std::memset(&segs, 0, sizeof(segs));
+    return quantize_impl(d_x, M, K, ld, d_g, segs, d_codes, d_sf, layout, info, as_stream(stream), kQuantRmsnorm,
+                         reinterpret_cast<const uint16_t*>(d_weight), eps);
 }
 
 size_t nvfp4_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int nseg) {

@@ -70,6 +70,13 @@ __device__ __forceinline__ void ldg256_stream(const void* p, uint32_t (&v)[8]) {
 
 // per 16-bit half: magnitude = max(|a|, |b|) (the sign bit of the result is sign(a) xor sign(b)
 // and is masked off by the caller)
+// 256-bit load that may stay in L1/L2 (data that is read again shortly)
+__device__ __forceinline__ void ldg256_cached(const void* p, uint32_t (&v)[8]) {
+    asm volatile("ld.global.nc.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+                 : "l"(p));
+}
+
 __device__ __forceinline__ uint32_t bf16x2_absmax(uint32_t a, uint32_t b) {
     uint32_t r;
     asm("max.xorsign.abs.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
@@ -141,13 +148,31 @@ __device__ __forceinline__ void swiglu_block(const uint32_t (&g)[8], const uint3
     }
 }
 
+// 16 values x and 16 weights w (packed bf16) -> bf16((x * rstd) * w), packed
+__device__ __forceinline__ void rmsnorm_block(const uint32_t (&x)[8], const uint32_t (&w)[8], float rstd, uint32_t (&y)[8]) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const float lo = __fmul_rn(__fmul_rn(__uint_as_float(x[i] << 16), rstd), __uint_as_float(w[i] << 16));
+        const float hi = __fmul_rn(__fmul_rn(__uint_as_float(x[i] & 0xFFFF0000u), rstd), __uint_as_float(w[i] & 0xFFFF0000u));
+        __nv_bfloat162 b2 = __floats2bfloat162_rn(lo, hi);
+        y[i] = *reinterpret_cast<uint32_t*>(&b2);
+    }
+}
+
+constexpr int kQuantPlain = 0, kQuantSwiglu = 1, kQuantRmsnorm = 2;
+
 // A warp owns `chunks_per_unit` consecutive 512-element chunks of one row (a "unit"); units are
 // dealt round-robin to a persistent grid.
-// SWIGLU: x is [M, 2K] (gate | up) and the tensor that is quantized is bf16(silu(gate) * up), [M, K].
-template <bool MMA_LAYOUT, int UNROLL, bool SWIGLU>
-__global__ void __launch_bounds__(256, SWIGLU ? 4 : 5)
+// MODE kQuantSwiglu: x is [M, 2K] (gate | up) and the tensor that is quantized is
+// bf16(silu(gate) * up), [M, K].  MODE kQuantRmsnorm: the quantized tensor is
+// bf16(x * rstd(row) * aux[k]) with rstd = 1 / sqrt(mean(x^2) + eps); a unit is then a whole row
+// (units_per_row == 1): the warp first sums the squares of its row (each lane over its own
+// 16-element pieces in increasing k, fused multiply-adds, then a butterfly over the 32 lanes),
+// and reads the row a second time, from cache, to normalise and quantize it.
+template <bool MMA_LAYOUT, int UNROLL, int MODE>
+__global__ void __launch_bounds__(256, MODE == kQuantPlain ? 5 : 4)
 quantize_kernel(const uint16_t* __restrict__ x, int32_t M, int32_t K, int64_t ld,
-                const float* __restrict__ g_ptr, SegTable segs,
+                const float* __restrict__ g_ptr, SegTable segs, const uint16_t* __restrict__ aux, float eps,
                 uint8_t* __restrict__ codes, uint8_t* __restrict__ sf,
                 int32_t chunks_per_row, int32_t chunks_per_unit, int32_t units_per_row, int32_t total_units) {
     const int lane = threadIdx.x & 31;
@@ -177,6 +202,26 @@ quantize_kernel(const uint16_t* __restrict__ x, int32_t M, int32_t K, int64_t ld
         uint8_t* sf_row = MMA_LAYOUT
             ? sf + static_cast<int64_t>(row >> 7) * katoms * 512 + (row & 31) * 16 + ((row & 127) >> 5) * 4
             : sf + static_cast<int64_t>(row) * KB;
+        float rstd = 0.0f;
+        if (MODE == kQuantRmsnorm) {
+            float ss = 0.0f;
+            for (int32_t c = 0; c < chunks_per_row; ++c) {
+                const int32_t k0 = c * 512 + lane * 16;
+                if (k0 < K) {
+                    uint32_t v[8];
+                    ldg256_cached(xrow + k0, v);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const float lo = __uint_as_float(v[i] << 16), hi = __uint_as_float(v[i] & 0xFFFF0000u);
+                        ss = __fmaf_rn(lo, lo, ss);
+                        ss = __fmaf_rn(hi, hi, ss);
+                    }
+                }
+            }
+#pragma unroll
+            for (int off = 16; off >= 1; off >>= 1) ss = __fadd_rn(ss, __shfl_xor_sync(0xffffffffu, ss, off));
+            rstd = __frcp_rn(__fsqrt_rn(__fadd_rn(__fdiv_rn(ss, static_cast<float>(K)), eps)));
+        }
         for (int32_t c0 = c_begin; c0 < c_end; c0 += UNROLL) {
             uint32_t v[UNROLL][8];
             int32_t col[UNROLL];
@@ -185,12 +230,19 @@ quantize_kernel(const uint16_t* __restrict__ x, int32_t M, int32_t K, int64_t ld
                 col[u] = (c0 + u < c_end) ? (c0 + u) * 512 + lane * 16 : K;
                 if (col[u] < K) {
                     ldg256_stream(xrow + col[u], v[u]);
-                    if (SWIGLU) {
+                    if (MODE == kQuantSwiglu) {
                         uint32_t up[8], h[8];
                         ldg256_stream(xrow + K + col[u], up);
                         swiglu_block(v[u], up, h);
 #pragma unroll
                         for (int i = 0; i < 8; ++i) v[u][i] = h[i];
+                    }
+                    if (MODE == kQuantRmsnorm) {
+                        uint32_t wv[8], y[8];
+                        ldg256_cached(aux + col[u], wv);
+                        rmsnorm_block(v[u], wv, rstd, y);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) v[u][i] = y[i];
                     }
                 } else {
 #pragma unroll

@@ -175,3 +175,31 @@ def test_swiglu_extreme_gates():
     torch.cuda.synchronize()
     codes_o, sf_o, _, _ = gu_mod.oracle_quantized(h, g=g)
     gu_mod.check_quantized(codes_d, sf_d, nv.SF_MMA, codes_o, sf_o, inner)
+
+
+# ---- producer fusion: RMSNorm(x) * w -> quantize in one pass ----------------------------------
+def _rmsnorm_case(M, K, layout=nv.SF_MMA, seed=12, eps=1e-6, ld_pad=0):
+    x = synth.prefill_activations(seed, 80, M, K)
+    w = synth.f64_to_bf16_bits(1.0 + 0.25 * np.cos(0.37 * np.arange(K)))
+    y = oracle.rmsnorm_bf16(x, w, eps)
+    _, g = oracle.calibrate(y)
+    t = gu_mod.dev_bf16(x)
+    if ld_pad:
+        buf = torch.zeros((M, K + ld_pad), dtype=torch.bfloat16, device=gu_mod.DEV)
+        buf[:, :K] = t
+        t = buf[:, :K]
+    codes_d, sf_d = nv.nvfp4_rmsnorm_quantize(t, gu_mod.dev_bf16(w), eps, gu_mod.dev_f32(g), layout)
+    torch.cuda.synchronize()
+    codes_o, sf_o, _, _ = gu_mod.oracle_quantized(y, g=g)
+    gu_mod.check_quantized(codes_d, sf_d, layout, codes_o, sf_o, K)
+
+
+@pytest.mark.parametrize("M,K", [(1, 16), (3, 528), (130, 5120), (64, 17408), (257, 1040)])
+@pytest.mark.parametrize("layout", [nv.SF_MMA, nv.SF_LINEAR])
+def test_rmsnorm_quantize_matches_oracle_composition(M, K, layout):
+    _rmsnorm_case(M, K, layout)
+
+
+def test_rmsnorm_quantize_strided_and_eps_zero():
+    _rmsnorm_case(40, 2048, ld_pad=32, eps=0.0)
+    _rmsnorm_case(2048, 5120, seed=13)
