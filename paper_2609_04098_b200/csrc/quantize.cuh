@@ -205,14 +205,24 @@ quantize_kernel(const uint16_t* __restrict__ x, int32_t M, int32_t K, int64_t ld
         float rstd = 0.0f;
         if (MODE == kQuantRmsnorm) {
             float ss = 0.0f;
-            for (int32_t c = 0; c < chunks_per_row; ++c) {
-                const int32_t k0 = c * 512 + lane * 16;
-                if (k0 < K) {
-                    uint32_t v[8];
-                    ldg256_cached(xrow + k0, v);
+            constexpr int PF = 4;                                   // loads in flight per lane
+            for (int32_t c = 0; c < chunks_per_row; c += PF) {
+                uint32_t v[PF][8];
+#pragma unroll
+                for (int u = 0; u < PF; ++u) {
+                    const int32_t k0 = (c + u) * 512 + lane * 16;
+                    if (k0 < K) {
+                        ldg256_cached(xrow + k0, v[u]);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) v[u][i] = 0u;   // adds +0: the sum is unchanged
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < PF; ++u) {
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
-                        const float lo = __uint_as_float(v[i] << 16), hi = __uint_as_float(v[i] & 0xFFFF0000u);
+                        const float lo = __uint_as_float(v[u][i] << 16), hi = __uint_as_float(v[u][i] & 0xFFFF0000u);
                         ss = __fmaf_rn(lo, lo, ss);
                         ss = __fmaf_rn(hi, hi, ss);
                     }
