@@ -439,30 +439,82 @@ def run_gpu(args):
         del xq, outs
 
     # ---- end to end: host buffers in, result back, through the same calls
-    e2e_steps = max(1, min(args.steps, 5))
-    h_out = torch.empty_like(d_result, device="cpu").pin_memory()
-    h2d_bytes = sum(t.numel() * t.element_size() for t in h2d_tensors)
-    d2h_bytes = h_out.numel() * h_out.element_size()
+    e2e_steps = max(4, min(args.steps, 20))
+    if args.workload == "mlp":
+        # The MLP as a caller runs it: X1 arrives from pinned host memory, the down projection's
+        # input is produced on the device (silu(gate)*up fused into the quantizer), Y comes back.
+        # Copies and compute are double-buffered over three streams, as a serving loop would do.
+        h_in = h2d_tensors[0]
+        xin = [x1, torch.empty_like(x1)]
+        yout = [y2, torch.empty_like(y2)]
+        h_outs = [torch.empty_like(y2, device="cpu").pin_memory() for _ in range(2)]
+        s_in, s_cmp, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
+        ev_in = [torch.cuda.Event() for _ in range(2)]
+        ev_cmp = [torch.cuda.Event() for _ in range(2)]
+        ev_out = [torch.cuda.Event() for _ in range(2)]
+        h2d_bytes = h_in.numel() * h_in.element_size()
+        d2h_bytes = h_outs[0].numel() * h_outs[0].element_size()
 
-    def e2e_step():
-        for src, dst in zip(h2d_tensors, d_inputs):
-            dst.copy_(src, non_blocking=True)
-        step()
-        h_out.copy_(d_result, non_blocking=True)
+        def pipelined(n):
+            for i in range(n):
+                b = i & 1
+                with torch.cuda.stream(s_in):
+                    s_in.wait_event(ev_cmp[b])                 # compute of step i-2 has read xin[b]
+                    xin[b].copy_(h_in, non_blocking=True)
+                    ev_in[b].record(s_in)
+                with torch.cuda.stream(s_cmp):
+                    s_cmp.wait_event(ev_in[b])
+                    s_cmp.wait_event(ev_out[b])                # the copy-out of step i-2 has read yout[b]
+                    nv.nvfp4_quantize_act(xin[b], g1, out=q1)
+                    nv.nvfp4_linear(q1[0], q1[1], g1, w_gu_c, w_gu_sf, wl.seg_gu, g_gu, ws, out=y1)
+                    nv.nvfp4_swiglu_quantize(y1, g2, out=q2)
+                    nv.nvfp4_linear(q2[0], q2[1], g2, w_d_c, w_d_sf, wl.seg_d, g_d, ws, out=yout[b])
+                    ev_cmp[b].record(s_cmp)
+                with torch.cuda.stream(s_out):
+                    s_out.wait_event(ev_cmp[b])
+                    h_outs[b].copy_(yout[b], non_blocking=True)
+                    ev_out[b].record(s_out)
 
-    e2e_step()
-    torch.cuda.synchronize()
-    barrier()
-    s0, s1 = ev(), ev()
-    s0.record(stream)
-    for _ in range(e2e_steps):
+        torch.cuda.synchronize()
+        pipelined(2)
+        torch.cuda.synchronize()
+        barrier()
+        s0, s1 = ev(), ev()
+        s0.record(stream)
+        for st_ in (s_in, s_cmp, s_out):
+            st_.wait_stream(stream)
+        pipelined(e2e_steps)
+        for st_ in (s_in, s_cmp, s_out):
+            stream.wait_stream(st_)
+        s1.record(stream)
+        torch.cuda.synchronize()
+        e2e_note = ("MLP with the fused producer (X1 from pinned host memory, Y back to host every step), "
+                    "copies and compute double-buffered over three streams")
+    else:
+        h_out = torch.empty_like(d_result, device="cpu").pin_memory()
+        h2d_bytes = sum(t.numel() * t.element_size() for t in h2d_tensors)
+        d2h_bytes = h_out.numel() * h_out.element_size()
+
+        def e2e_step():
+            for src, dst in zip(h2d_tensors, d_inputs):
+                dst.copy_(src, non_blocking=True)
+            step()
+            h_out.copy_(d_result, non_blocking=True)
+
         e2e_step()
-    s1.record(stream)
-    torch.cuda.synchronize()
+        torch.cuda.synchronize()
+        barrier()
+        s0, s1 = ev(), ev()
+        s0.record(stream)
+        for _ in range(e2e_steps):
+            e2e_step()
+        s1.record(stream)
+        torch.cuda.synchronize()
+        e2e_note = "host input in, fused call, result back, on one stream"
     e2e_ms = group.max_over_ranks(s0.elapsed_time(s1) / e2e_steps)
     result["e2e"] = {"value": round(wl.flops * world / (e2e_ms * 1e-3) / 1e12, 2), "unit": "TFLOP/s",
                      "ms_per_step": round(e2e_ms, 3), "h2d_bytes_per_step": h2d_bytes,
-                     "d2h_bytes_per_step": d2h_bytes}
+                     "d2h_bytes_per_step": d2h_bytes, "what": e2e_note}
     status = nv.device_status(ws if args.workload == "mlp" else wss[0])
     if status != 0:
         raise SystemExit("device status %d after the timed region" % status)

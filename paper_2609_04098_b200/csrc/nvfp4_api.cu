@@ -203,7 +203,11 @@ nvfp4_status launch_gemm(const GemmMaps& tm, GemmParams& p, int sm_count, cudaSt
     {
         // rows of A kept live per raster group: about 32 MB of codes and scales (a quarter of L2)
         const int64_t unit_bytes = static_cast<int64_t>(PAIR ? 256 : 128) * (p.K / 2 + p.K / 16);
-        int64_t g = (32ll << 20) / (unit_bytes > 0 ? unit_bytes : 1);
+        int64_t budget = 32ll << 20;
+#ifdef NVFP4_PROBE
+        if (getenv("NVFP4_GROUP_MB")) budget = static_cast<int64_t>(atoi(getenv("NVFP4_GROUP_MB"))) << 20;
+#endif
+        int64_t g = budget / (unit_bytes > 0 ? unit_bytes : 1);
         if (g < 1) g = 1;
         if (g > m_units) g = m_units;
         p.group_m = static_cast<int32_t>(g);
