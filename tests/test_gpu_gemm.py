@@ -246,3 +246,67 @@ def test_small_m_split_k(M, N, K, out_f32):
     # and the one-tile-per-CTA kernel gives the same answer (within summation order)
     y1 = _run_from_oracle_operands(segs, ac, asf, ga, wc, wsf, gs, K, out_f32=out_f32)    # 256-byte workspace: no split
     gu.check_gemm(y1, y_ref, bound, "no split")
+
+
+# ---- the benchmark's own shapes at full size (whole device path, auto tile choice) ------------
+def _full_size_sampled(M, K, spec, seed, n_rows=16, n_cols=24):
+    """Device path end to end (calibrate, quantize, GEMM) at full size; the oracle checks the
+    quantized operands in full, the GEMM on sampled rows, sampled columns (every segment edge and
+    the last column among them) and a random-sign projection of the whole output."""
+    segs = synth.make_segments(spec)
+    N = sum(s.count for s in segs)
+    x = synth.prefill_activations(seed, 501, M, K)
+    w = synth.weights(seed, 502, segs, K)
+    ac, asf, ga, _ = gu.oracle_quantized(x)
+    wc, wsf, gs, _ = gu.oracle_quantized(w, segments=segs)
+    gcol = oracle.col_scales(N, segs, gs)
+    xt, wt = gu.dev_bf16(x), gu.dev_bf16(w)
+    g_a = nv.nvfp4_calibrate(xt)
+    a_codes, a_sf = nv.nvfp4_quantize_act(xt, g_a)
+    w_codes, w_sf, g_seg = nv.nvfp4_quantize_weight(wt, segs)
+    del xt, wt
+    gu.check_quantized(a_codes, a_sf, nv.SF_MMA, ac, asf, K)
+    gu.check_quantized(w_codes, w_sf, nv.SF_MMA, wc, wsf, K)
+    ws = _ws()
+    y = nv.nvfp4_linear(a_codes, a_sf, g_a, w_codes, w_sf, segs, g_seg, ws)
+    assert nv.device_status(ws) == 0
+    rng = np.random.default_rng(seed)
+    step = max(1, (M // 128) // n_rows)
+    rows = np.unique(np.array([t * 128 + rng.integers(0, 128) for t in range(0, M // 128, step)] + [0, M - 1]))
+    y_rows = oracle.gemm(ac, asf, ga, wc, wsf, gcol, rows=rows)
+    gu.check_gemm(y[torch.from_numpy(rows).to(gu.DEV)], y_rows,
+                  gu.gemm_bounds(ac, asf, ga, wc, wsf, gcol, rows=rows), "rows")
+    edge = {c for s in segs for c in (s.begin, s.begin + s.count - 1)} | {0, N - 1}
+    cols = np.array(sorted(edge | set(rng.integers(0, N, n_cols).tolist())))
+    y_cols = oracle.gemm(ac, asf, ga, wc, wsf, gcol, cols=cols)
+    gu.check_gemm(y[:, torch.from_numpy(cols).to(gu.DEV)].contiguous(), y_cols,
+                  gu.gemm_bounds(ac, asf, ga, wc, wsf, gcol, cols=cols), "cols")
+    # projection of the whole output on a random sign vector, operands dequantized in row chunks
+    r = rng.choice([-1.0, 1.0], N)
+    wr = np.zeros(K)
+    w_norm2 = 0.0
+    for b in range(0, N, 4096):
+        w_hat = oracle.dequantize(wc[b:b + 4096], wsf[b:b + 4096], gcol[b:b + 4096])
+        wr += w_hat.T @ r[b:b + 4096]
+        w_norm2 += float((w_hat ** 2).sum())
+    worst = 0.0
+    r_dev = torch.from_numpy(r).to(gu.DEV)
+    got = (y.double() @ r_dev).cpu().numpy()
+    for b in range(0, M, 2048):
+        a_hat = oracle.dequantize(ac[b:b + 2048], asf[b:b + 2048], oracle.row_scales(min(2048, M - b), g=ga))
+        want = a_hat @ wr
+        scale = np.linalg.norm(a_hat, axis=1) * np.sqrt(w_norm2) / np.sqrt(K)
+        worst = max(worst, float(np.max(np.abs(got[b:b + 2048] - want) / scale)))
+    assert worst < 2e-2, worst
+
+
+def test_mlp_gate_up_full_size_sampled():
+    _full_size_sampled(8192, synth.HIDDEN, (("gate", synth.MLP_INNER, 0.02), ("up", synth.MLP_INNER, 0.02)), 1)
+
+
+def test_mlp_down_full_size_sampled():
+    _full_size_sampled(8192, synth.MLP_INNER, (("down", synth.HIDDEN, 0.02),), 2)
+
+
+def test_long_prefill_32k_tokens_sampled():
+    _full_size_sampled(32768, synth.HIDDEN, (("w", 6144, 0.02),), 3, n_rows=32)
