@@ -184,6 +184,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     if (PAIR) ptx::cluster_sync_all(); else __syncthreads();   // barriers and TMEM exist from here on
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // Everything above ran while the kernel in front of this one (the activation quantizer, which
+    // releases its dependents early) may still have been working; nothing below may read global
+    // memory before that kernel has finished.
+    ptx::pdl_wait();
 
     // tile index -> (row unit, column tile).  Tiles are visited in groups of `group_m` row
     // units; inside a group the row unit varies fastest, then the column tile.  The CTAs that

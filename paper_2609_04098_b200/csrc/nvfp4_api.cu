@@ -214,16 +214,20 @@ nvfp4_status launch_gemm(const GemmMaps& tm, GemmParams& p, int sm_count, cudaSt
     }
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof(cfg));
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = PAIR ? 2 : 1;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    // may start while the quantize kernel in front of it still runs (that kernel says when);
+    // only the loads of its output wait for it
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.blockDim = dim3(kGemmThreads, 1, 1);
     cfg.dynamicSmemBytes = C::SMEM_BYTES;
     cfg.stream = stream;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     int units = 0;
     {
         std::lock_guard<std::mutex> lock(mu);
@@ -296,20 +300,15 @@ nvfp4_status quantize_impl(const void* d_x, int64_t M, int64_t K, int64_t ld, co
                            const uint16_t* aux = nullptr, float eps = 0.0f) {
     const int64_t chunks = (K + 511) / 512;              // 512 elements = one block per lane
     if (M >= (1ll << 31) || K >= (1ll << 31)) return NVFP4_ERR_SHAPE;
-    if (layout == NVFP4_SF_MMA && (M % 128) != 0) {
-        // rows of the last 128-row band that the tensor does not have must read as zero scales
-        const int64_t katoms = (K / 16 + 3) / 4;
-        if (cudaMemsetAsync(d_sf + (M / 128) * katoms * 512, 0, static_cast<size_t>(katoms * 512), stream) !=
-            cudaSuccess)
-            return NVFP4_ERR_CUDA;
-    }
     // a unit = up to `per_unit` consecutive chunks of one row, handled by one warp
     constexpr int kUnroll = 2;      // matches launch_quantize
     const int64_t resident_warps = static_cast<int64_t>(info.sm_count) * 40;   // 5 blocks of 8 warps per SM
     int64_t per_unit = (M * chunks > 2 * resident_warps) ? kUnroll : 1;
     if (mode == kQuantRmsnorm) per_unit = chunks;           // the row reduction needs the whole row in one warp
     const int64_t units_per_row = (chunks + per_unit - 1) / per_unit;
-    const int64_t units = M * units_per_row;
+    // in the tensor-core layout the kernel also zero-fills the scales of the rows that pad the last band
+    const int64_t rows_total = (layout == NVFP4_SF_MMA) ? (M + 127) / 128 * 128 : M;
+    const int64_t units = rows_total * units_per_row;
     if (units >= (1ll << 31)) return NVFP4_ERR_SHAPE;
     const uint16_t* x = reinterpret_cast<const uint16_t*>(d_x);
     const bool mma = layout == NVFP4_SF_MMA;

@@ -88,6 +88,19 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
     }
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// primary side: kernels launched behind this one (with the programmatic-serialization attribute)
+// may start now; what they need from this kernel they get after their own pdl_wait()
+__device__ __forceinline__ void pdl_launch_dependents() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+// secondary side: returns once the kernels this launch depends on have completed and their
+// writes are visible (a no-op for a normal launch)
+__device__ __forceinline__ void pdl_wait() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("fence.proxy.async;" ::: "memory");
+}
+
 // ---------------------------------------------------------------- clusters
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;

@@ -13,6 +13,7 @@
 #include <cuda_runtime.h>
 
 #include "../../include/nvfp4.h"
+#include "ptx.cuh"
 
 namespace nvfp4 {
 
@@ -175,6 +176,9 @@ quantize_kernel(const uint16_t* __restrict__ x, int32_t M, int32_t K, int64_t ld
                 const float* __restrict__ g_ptr, SegTable segs, const uint16_t* __restrict__ aux, float eps,
                 uint8_t* __restrict__ codes, uint8_t* __restrict__ sf,
                 int32_t chunks_per_row, int32_t chunks_per_unit, int32_t units_per_row, int32_t total_units) {
+    // the GEMM that consumes this tensor may start its prologue and its weight loads now; it
+    // waits for this kernel's completion before it touches the codes and scales written here
+    ptx::pdl_launch_dependents();
     const int lane = threadIdx.x & 31;
     const int32_t warp_global = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int32_t nwarps = gridDim.x * (blockDim.x >> 5);
@@ -190,6 +194,17 @@ quantize_kernel(const uint16_t* __restrict__ x, int32_t M, int32_t K, int64_t ld
         if (part >= units_per_row) { part -= units_per_row; ++row; }
         const int32_t c_begin = part * chunks_per_unit;
         const int32_t c_end = min(chunks_per_row, c_begin + chunks_per_unit);
+        if (row >= M) {
+            // tensor-core layout only: rows that pad the last 128-row band get zero scales
+            if (MMA_LAYOUT) {
+                uint8_t* pad_row = sf + static_cast<int64_t>(row >> 7) * katoms * 512 + (row & 31) * 16 + ((row & 127) >> 5) * 4;
+                for (int32_t c = c_begin; c < c_end; ++c) {
+                    const int32_t kb = c * 32 + lane;
+                    if ((lane & 3) == 0 && kb < KB) *reinterpret_cast<uint32_t*>(pad_row + static_cast<int64_t>(kb >> 2) * 512) = 0u;
+                }
+            }
+            continue;
+        }
         float g = g_single, c1 = c1_single;
         if (segs.nseg != 0) {
             g = __ldg(g_ptr + seg_of(segs, row));
