@@ -208,6 +208,10 @@ size_t nvfp4_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int nseg);
  * (paper: Section 9, "Decode overhead" -- activation quantization is the overhead
  * that matters at small batch), codes and scales live in the workspace.
  *   d_x   bf16 [M, K], row stride ldx, 32-byte aligned, ldx % 16 == 0
+ * For M = 1 or 2 (single-stream decode) the call is one weight-streaming kernel on the CUDA cores
+ * that quantizes the activations itself (same codes) and does not touch the workspace; from M = 3
+ * on it is the quantize kernel followed by the tensor-core GEMM, which starts its prologue while
+ * the quantizer still runs.
  */
 nvfp4_status nvfp4_linear_bf16(const void* d_x, int64_t ldx, const float* d_g_a,
                                int64_t M, int64_t K,

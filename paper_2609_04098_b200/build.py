@@ -13,7 +13,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libnvfp4_b200.so")
 SOURCES = ["nvfp4_api.cu"]
-HEADERS = ["gemm.cuh", "quantize.cuh", "ptx.cuh", os.path.join("..", "..", "include", "nvfp4.h")]
+HEADERS = ["gemm.cuh", "decode.cuh", "quantize.cuh", "ptx.cuh", os.path.join("..", "..", "include", "nvfp4.h")]
 
 
 def nvcc_path() -> str:

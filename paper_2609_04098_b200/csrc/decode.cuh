@@ -1,0 +1,224 @@
+// Decode-sized batches (1 or 2 tokens): the linear layer is a weight-streaming problem, bound by
+// HBM/L2 bandwidth and launch latency, not by the tensor cores -- a tile of 128 token rows would
+// be almost all padding.  One kernel, no tensor memory, no TMA pipeline:
+//   1. every CTA quantizes the few activation rows itself (same block arithmetic as
+//      quantize_kernel, so the codes are the ones the oracle produces) and keeps them in shared
+//      memory as exact fp16 values (E2M1 values need 3 bits) plus one float scale per block;
+//   2. each warp streams whole weight rows: a lane takes 32 consecutive codes (two blocks) per
+//      1024-element slice, decodes them to fp16, multiplies with the activation values
+//      (products and 8-term partial sums are exact in fp16), adds the two halves in fp32, scales
+//      the block sum by e4m3(s_a) * e4m3(s_w) (exact in fp32) and accumulates in fp32;
+//   3. a warp shuffle adds the 32 lane sums; lane 0 applies g_a * g_seg[segment] and stores.
+// The result differs from the exact product only by fp32 accumulation rounding.
+#pragma once
+#include <cstdint>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include "../../include/nvfp4.h"
+#include "quantize.cuh"
+
+namespace nvfp4 {
+
+struct DecodeParams {
+    const uint16_t* x;       // bf16 [M, K], row stride ldx
+    int64_t ldx;
+    const float* g_a;
+    const uint8_t* w_codes;  // [N, K/2]
+    const uint8_t* w_sf;     // tensor-core scale layout
+    const float* g_seg;
+    void* y;
+    int64_t ldy;
+    int32_t M, N, K;
+    uint32_t flags;
+    int32_t nseg;
+    int32_t seg_end[NVFP4_MAX_SEGMENTS];
+};
+
+constexpr int kDecodeThreads = 512;
+constexpr int kDecodeSlices = 5;              // 1024-element slices of a weight row in flight per lane
+
+// eight packed E2M1 codes (one 32-bit word, element i in nibble i) -> four half2 (element 2j in .x)
+__device__ __forceinline__ void e2m1x8_to_half2x4(uint32_t w, __half2 (&out)[4]) {
+    uint32_t h0, h1, h2, h3;
+    asm("{\n\t"
+        ".reg .b8 b0, b1, b2, b3;\n\t"
+        "mov.b32 {b0, b1, b2, b3}, %4;\n\t"
+        "cvt.rn.f16x2.e2m1x2 %0, b0;\n\t"
+        "cvt.rn.f16x2.e2m1x2 %1, b1;\n\t"
+        "cvt.rn.f16x2.e2m1x2 %2, b2;\n\t"
+        "cvt.rn.f16x2.e2m1x2 %3, b3;\n\t"
+        "}\n"
+        : "=r"(h0), "=r"(h1), "=r"(h2), "=r"(h3)
+        : "r"(w));
+    out[0] = *reinterpret_cast<__half2*>(&h0);
+    out[1] = *reinterpret_cast<__half2*>(&h1);
+    out[2] = *reinterpret_cast<__half2*>(&h2);
+    out[3] = *reinterpret_cast<__half2*>(&h3);
+}
+
+// activation values per token: whole 1024-element slices, stored so that the 16-byte piece a lane
+// reads next to its neighbours' is contiguous with theirs: element k = 1024 s + 32 lane + 8 q + e
+// lives at half index ((4 s + q) * 32 + lane) * 8 + e   (bank-conflict-free 128-bit reads)
+inline size_t decode_kpad(int64_t K) { return static_cast<size_t>((K + 1023) / 1024 * 1024); }
+inline size_t decode_smem_bytes(int64_t M, int64_t K) {
+    return static_cast<size_t>(M) * decode_kpad(K) * 2 + static_cast<size_t>(M) * static_cast<size_t>(K / 16) * 4;
+}
+
+template <int MT>
+__global__ void __launch_bounds__(kDecodeThreads, 1)
+decode_gemv_kernel(const __grid_constant__ DecodeParams p) {
+    extern __shared__ __align__(16) uint8_t dsm[];
+    const int K = p.K, KB = K >> 4;
+    const int KP = ((K + 1023) >> 10) << 10;
+    __half* a_val = reinterpret_cast<__half*>(dsm);                                   // [MT][KP], permuted
+    float* a_scale = reinterpret_cast<float*>(dsm + static_cast<size_t>(MT) * KP * 2);    // [MT][K/16]
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+
+    // ---- weight streaming set-up; the first item's loads are issued before the activations are
+    // quantized so that their latency overlaps that work
+    const int katoms = (KB + 3) >> 2;
+    const int n_slices = (K + 1023) >> 10;
+    const int warps_total = gridDim.x * (kDecodeThreads >> 5);
+    const bool out_f32 = (p.flags & NVFP4_OUT_F32) != 0u;
+    // a warp's work is a flat list of (row, group of kDecodeSlices slices); the loads of the next
+    // item are issued before the current one is consumed, so the memory latency is paid once
+    const int groups = (n_slices + kDecodeSlices - 1) / kDecodeSlices;
+    const int first_row = blockIdx.x * (kDecodeThreads >> 5) + warp;
+    const int my_rows = first_row < p.N ? (p.N - first_row + warps_total - 1) / warps_total : 0;
+    const int items = my_rows * groups;
+    uint4 wv[2][kDecodeSlices];
+    uint32_t sfw[2][kDecodeSlices];
+    auto load_item = [&](int item, int buf) {
+        const int r = item / groups, s0 = (item - r * groups) * kDecodeSlices;
+        const int n = first_row + r * warps_total;
+        const uint8_t* wrow = p.w_codes + static_cast<int64_t>(n) * (K >> 1);
+        const uint8_t* sfrow = p.w_sf + static_cast<int64_t>(n >> 7) * katoms * 512 + (n & 31) * 16 + ((n & 127) >> 5) * 4;
+#pragma unroll
+        for (int u = 0; u < kDecodeSlices; ++u) {
+            const int k0 = (s0 + u) * 1024 + lane * 32;                     // this lane's 32 codes
+            wv[buf][u] = make_uint4(0u, 0u, 0u, 0u);
+            sfw[buf][u] = 0u;
+            if (s0 + u < n_slices && k0 < K) {
+                wv[buf][u] = __ldcs(reinterpret_cast<const uint4*>(wrow + (k0 >> 1)));
+                const int kb = k0 >> 4;                                      // even: both scale bytes sit in one word
+                sfw[buf][u] = *reinterpret_cast<const uint16_t*>(sfrow + static_cast<int64_t>(kb >> 2) * 512 + (kb & 3));
+            }
+        }
+    };
+    if (items > 0) load_item(0, 0);
+
+    // ---- 1. quantize the activation rows (every CTA its own copy)
+    {
+        const float g = __ldg(p.g_a);
+        const float c1 = __fdiv_rn(1.0f, __fmul_rn(6.0f, g));
+        for (int b = threadIdx.x; b < MT * KB; b += kDecodeThreads) {
+            const int m = b / KB, kb = b - m * KB;
+            uint32_t v[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+            if (m < p.M) ldg256_cached(p.x + static_cast<int64_t>(m) * p.ldx + kb * 16, v);
+            uint32_t s8;
+            const uint2 codes = quantize_block(v, g, c1, s8);
+            a_scale[m * KB + kb] = e4m3_to_f32(s8);
+            const int k0 = kb * 16, sl = k0 >> 10, ln = (k0 & 1023) >> 5, q0 = (k0 & 31) >> 3;
+            __half* base = a_val + static_cast<size_t>(m) * KP;
+            __half2 lo[4], hi[4];
+            e2m1x8_to_half2x4(codes.x, lo);
+            e2m1x8_to_half2x4(codes.y, hi);
+            *reinterpret_cast<uint4*>(base + ((sl * 4 + q0) * 32 + ln) * 8) = *reinterpret_cast<uint4*>(lo);
+            *reinterpret_cast<uint4*>(base + ((sl * 4 + q0 + 1) * 32 + ln) * 8) = *reinterpret_cast<uint4*>(hi);
+        }
+    }
+    __syncthreads();
+
+    // ---- 2. stream weight rows
+    float acc[MT];
+#pragma unroll 1
+    for (int item = 0; item < items; ++item) {
+        const int buf = item & 1;
+        const int r = item / groups, g0 = item - r * groups, s0 = g0 * kDecodeSlices;
+        const int n = first_row + r * warps_total;
+        if (item + 1 < items) {
+            if (buf == 0) load_item(item + 1, 1); else load_item(item + 1, 0);
+        }
+        if (g0 == 0) {
+#pragma unroll
+            for (int m = 0; m < MT; ++m) acc[m] = 0.0f;
+        }
+        {
+#pragma unroll
+            for (int u = 0; u < kDecodeSlices; ++u) {
+                const int k0 = (s0 + u) * 1024 + lane * 32;
+                if (!(s0 + u < n_slices && k0 < K)) continue;
+                const uint4 wcur = buf == 0 ? wv[0][u] : wv[1][u];
+                const uint32_t scur = buf == 0 ? sfw[0][u] : sfw[1][u];
+                // weight scales of the two blocks, weight values as half2
+                uint32_t sh2;
+                asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(sh2) : "h"(static_cast<uint16_t>(scur)));
+                const float2 sw = __half22float2(*reinterpret_cast<__half2*>(&sh2));
+                __half2 wq[16];
+                {
+                    __half2 t[4];
+                    e2m1x8_to_half2x4(wcur.x, t);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) wq[j] = t[j];
+                    e2m1x8_to_half2x4(wcur.y, t);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) wq[4 + j] = t[j];
+                    e2m1x8_to_half2x4(wcur.z, t);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) wq[8 + j] = t[j];
+                    e2m1x8_to_half2x4(wcur.w, t);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) wq[12 + j] = t[j];
+                }
+                const int kb = k0 >> 4;
+#pragma unroll
+                for (int m = 0; m < MT; ++m) {
+                    // piece q of this lane: 32 lanes x 16 bytes apart from piece q + 1
+                    const uint4* ap = reinterpret_cast<const uint4*>(a_val + static_cast<size_t>(m) * KP) +
+                                      (static_cast<size_t>(s0 + u) * 4) * 32 + lane;
+                    __half2 s0h = __float2half2_rn(0.0f), s1h = __float2half2_rn(0.0f);
+#pragma unroll
+                    for (int q = 0; q < 2; ++q) {                            // block 0: 8 half2
+                        const uint4 av = ap[q * 32];
+                        const __half2* a2 = reinterpret_cast<const __half2*>(&av);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) s0h = __hfma2(a2[e], wq[4 * q + e], s0h);
+                    }
+#pragma unroll
+                    for (int q = 2; q < 4; ++q) {                            // block 1
+                        const uint4 av = ap[q * 32];
+                        const __half2* a2 = reinterpret_cast<const __half2*>(&av);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) s1h = __hfma2(a2[e], wq[4 * q + e], s1h);
+                    }
+                    const float2 b0 = __half22float2(s0h), b1 = __half22float2(s1h);
+                    const float2 sa = *reinterpret_cast<const float2*>(a_scale + m * KB + kb);     // kb is even
+                    acc[m] = __fmaf_rn(__fadd_rn(b0.x, b0.y), __fmul_rn(sa.x, sw.x), acc[m]);
+                    acc[m] = __fmaf_rn(__fadd_rn(b1.x, b1.y), __fmul_rn(sa.y, sw.y), acc[m]);
+                }
+            }
+        }
+        if (g0 + 1 < groups) continue;                     // more slices of this row to come
+        // ---- 3. reduce over lanes, scale, store
+#pragma unroll
+        for (int m = 0; m < MT; ++m)
+#pragma unroll
+            for (int off = 16; off >= 1; off >>= 1) acc[m] += __shfl_xor_sync(0xffffffffu, acc[m], off);
+        if (lane == 0) {
+            int sgi = 0;
+            while (sgi + 1 < p.nseg && n >= p.seg_end[sgi]) ++sgi;
+            const float alpha = __fmul_rn(__ldg(p.g_a), __ldg(p.g_seg + sgi));
+#pragma unroll
+            for (int m = 0; m < MT; ++m) {
+                if (m >= p.M) break;
+                const float v = __fmul_rn(acc[m], alpha);
+                if (out_f32) reinterpret_cast<float*>(p.y)[static_cast<int64_t>(m) * p.ldy + n] = v;
+                else reinterpret_cast<__nv_bfloat16*>(p.y)[static_cast<int64_t>(m) * p.ldy + n] = __float2bfloat16_rn(v);
+            }
+        }
+    }
+}
+
+}  // namespace nvfp4

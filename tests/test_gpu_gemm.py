@@ -310,3 +310,34 @@ def test_mlp_down_full_size_sampled():
 
 def test_long_prefill_32k_tokens_sampled():
     _full_size_sampled(32768, synth.HIDDEN, (("w", 6144, 0.02),), 3, n_rows=32)
+
+
+# ---- 1 or 2 tokens: the weight-streaming decode kernel behind nvfp4_linear_bf16 (3, 4: tensor cores) ------------------
+@pytest.mark.parametrize("M", [1, 2, 3, 4])
+@pytest.mark.parametrize("N,K", [(6144, 5120), (1000, 1088), (5120, 17408), (50, 64)])
+@pytest.mark.parametrize("out_f32", [False, True])
+def test_decode_batches(M, N, K, out_f32):
+    n1 = max(1, N // 3)
+    segs = synth.make_segments((("p", n1, 0.02), ("q", N - n1, 0.2)))
+    x = synth.activations(19, 1, M, K, n_hot=2, hot_scale=50.0)
+    w = synth.weights(19, 2, segs, K)
+    ac, asf, ga, _ = gu.oracle_quantized(x)
+    wc, wsf, gs, _ = gu.oracle_quantized(w, segments=segs)
+    gcol = oracle.col_scales(N, segs, gs)
+    y_ref = oracle.gemm(ac, asf, ga, wc, wsf, gcol)
+    ws = nv.alloc_workspace(gu.DEV, M, N, K, 2, fused=True)
+    launches = nv.launch_count()
+    y = nv.nvfp4_linear_bf16(gu.dev_bf16(x), gu.dev_f32(ga), gu.dev_u8(wc), gu.dev_u8(oracle.sf_to_mma(wsf, K)), segs,
+                             gu.dev_f32(gs), ws, out_f32=out_f32)
+    torch.cuda.synchronize()
+    assert nv.launch_count() - launches == (1 if M <= 2 else 2)     # 1-2 tokens: one kernel, quantization included
+    gu.check_gemm(y, y_ref, gu.gemm_bounds(ac, asf, ga, wc, wsf, gcol), "decode %s" % ((M, N, K),))
+    if out_f32 and M <= 2:
+        # no output rounding and exact block sums: only fp32 accumulation order separates it from the oracle
+        assert np.max(np.abs(y.cpu().numpy().astype(np.float64) - y_ref)) <= 2e-6 * np.max(np.abs(y_ref)) + 1e-30
+    # the tensor-core path (forced) agrees within the same bounds
+    nv.set_gemm_variant(128)
+    y2 = nv.nvfp4_linear_bf16(gu.dev_bf16(x), gu.dev_f32(ga), gu.dev_u8(wc), gu.dev_u8(oracle.sf_to_mma(wsf, K)), segs,
+                              gu.dev_f32(gs), ws, out_f32=out_f32)
+    nv.set_gemm_variant(0)
+    gu.check_gemm(y2, y_ref, gu.gemm_bounds(ac, asf, ga, wc, wsf, gcol), "tensor-core path")
