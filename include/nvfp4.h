@@ -175,6 +175,20 @@ nvfp4_status nvfp4_harmonize_scales(const uint8_t* d_sf_in, int64_t N, int64_t K
                                     uint8_t* d_sf_out, float* d_g_shared, void* stream);
 
 /*
+ * Statistics of a bf16 tensor at NVFP4 granularity (paper: Table "stats" -- max/RMS, kurtosis,
+ * share of "1-hot" 16-element blocks with max/RMS > 3, relative error of quantizing the tensor
+ * alone).  Writes seven doubles to d_out (8-byte aligned device memory):
+ *   [0] sum x^2   [1] sum x^4   [2] sum (x - dequant(quant(x)))^2   [3] max |x|
+ *   [4] number of blocks   [5] number of 1-hot blocks   [6] scratch
+ * from which  max/RMS = [3] / sqrt([0]/n),  kurtosis = n [1] / [0]^2,  1-hot share = [5]/[4],
+ * error = sqrt([2]/[0]).  Per-block sums are binary32 in a fixed order, blocks are added in double
+ * by atomics (the last bits depend on arrival order).
+ *   d_x  bf16 [rows, cols], row stride ld; 32-byte aligned, ld % 16 == 0, cols % 16 == 0;  d_g as usual
+ */
+nvfp4_status nvfp4_tensor_stats(const void* d_x, int64_t rows, int64_t cols, int64_t ld, const float* d_g,
+                                double* d_out, void* stream);
+
+/*
  * The W4A4 linear layer (paper: Background, "NVFP4": the GEMM runs on 4-bit tensor
  * cores; Section 6: per-module global scales meeting in one fused GEMM -- here each
  * segment of output columns gets its own global scale in the epilogue, which is

@@ -72,6 +72,8 @@ def _load():
     L.orc_dequantize.argtypes = [u8p, u8p, f32p, i64, i64, f64p]
     L.orc_harmonize_scales.restype = ctypes.c_float
     L.orc_harmonize_scales.argtypes = [u8p, i64, i64, f32p, u8p]
+    L.orc_stats.restype = ctypes.c_int
+    L.orc_stats.argtypes = [u16p, i64, i64, i64, ctypes.c_float, f64p]
     L.orc_sf_mma_bytes.restype = i64
     L.orc_sf_mma_bytes.argtypes = [i64, i64]
     L.orc_sf_mma_index.restype = i64
@@ -208,6 +210,31 @@ def harmonize_scales(sf_linear: np.ndarray, g_row: np.ndarray):
     out = np.empty_like(sf)
     gstar = _load().orc_harmonize_scales(_p(sf), sf.shape[0], sf.shape[1], _p(g_row), _p(out))
     return out, np.float32(gstar)
+
+
+def derive_stats(raw, n_elements: int) -> dict:
+    """{sum x^2, sum x^4, sum err^2, amax, blocks, 1-hot blocks} -> the table's columns."""
+    s2, s4, se, amax, nb, hot = [float(v) for v in raw]
+    rms = (s2 / n_elements) ** 0.5 if n_elements else 0.0
+    return {"max_over_rms": amax / rms if rms > 0 else 0.0,
+            "kurtosis": n_elements * s4 / (s2 * s2) if s2 > 0 else 0.0,
+            "onehot_share": hot / nb if nb else 0.0,
+            "rel_error": (se / s2) ** 0.5 if s2 > 0 else 0.0}
+
+
+def stats_raw(x_bits: np.ndarray, g) -> np.ndarray:
+    x = _c(x_bits, np.uint16)
+    out = np.zeros(6, np.float64)
+    rc = _load().orc_stats(_p(x), x.shape[0], x.shape[1], x.shape[1], ctypes.c_float(float(np.float32(g))), _p(out))
+    if rc != 0:
+        raise ValueError("columns must be a multiple of 16")
+    return out
+
+
+def stats(x_bits: np.ndarray, g) -> dict:
+    """max/RMS, kurtosis, 1-hot block share and quantization error of a bf16 tensor at NVFP4 granularity."""
+    x = _c(x_bits, np.uint16)
+    return derive_stats(stats_raw(x, g), x.size)
 
 
 def sf_mma_bytes(rows: int, cols: int) -> int:

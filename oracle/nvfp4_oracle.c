@@ -277,6 +277,50 @@ void orc_dequantize(const uint8_t* codes, const uint8_t* sf, const float* g_row,
 }
 
 /* ------------------------------------------------------------------------- */
+/* Statistics at NVFP4 granularity (the columns of the paper's Table "stats"): */
+/* max/RMS, kurtosis, share of "1-hot" blocks (block max/RMS > 3, i.e. one     */
+/* value holds more than 9/16 of the block's energy) and the relative error of */
+/* quantizing the tensor alone.  Per block, in binary32 (fmaf fused):          */
+/*   s2 = sum fmaf(x,x,.)   s4 = sum fmaf(x*x, x*x, .)   1-hot: bmax*bmax*16 > 9*s2 */
+/*   se = sum fmaf(e,e,.), e = x - e2m1(code) * (e4m3(s8) * g)                  */
+/* Block results are added up in double.  out: {sum x^2, sum x^4, sum err^2,   */
+/* amax, blocks, 1-hot blocks}.                                                */
+/* ------------------------------------------------------------------------- */
+int orc_stats(const uint16_t* x, int64_t rows, int64_t cols, int64_t ld, float g, double* out) {
+    if (cols % 16 != 0) return 1;
+    double t2 = 0.0, t4 = 0.0, te = 0.0, hot = 0.0;
+    float amax = 0.0f;
+    const float c1 = 1.0f / (6.0f * g);
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t b = 0; b < cols / 16; ++b) {
+            const uint16_t* xb = x + r * ld + b * 16;
+            float s2 = 0.0f, s4 = 0.0f, se = 0.0f, bmax = 0.0f;
+            for (int i = 0; i < 16; ++i) {
+                const float v = bf16_to_f32(xb[i]);
+                const float q = v * v;
+                s2 = fmaf(v, v, s2);
+                s4 = fmaf(q, q, s4);
+                if (fabsf(v) > bmax) bmax = fabsf(v);
+            }
+            if (bmax > amax) amax = bmax;
+            if ((bmax * bmax) * 16.0f > 9.0f * s2) hot += 1.0;
+            const uint8_t s8 = orc_e4m3_encode(bmax * c1);
+            const float d = orc_e4m3_decode(s8) * g;
+            const float qinv = 1.0f / d;
+            for (int i = 0; i < 16; ++i) {
+                const float v = bf16_to_f32(xb[i]);
+                const float xh = (s8 == 0) ? 0.0f : orc_e2m1_decode(orc_e2m1_encode(v * qinv)) * d;
+                const float e = v - xh;
+                se = fmaf(e, e, se);
+            }
+            t2 += (double)s2; t4 += (double)s4; te += (double)se;
+        }
+    out[0] = t2; out[1] = t4; out[2] = te; out[3] = (double)amax;
+    out[4] = (double)(rows * (cols / 16)); out[5] = hot;
+    return 0;
+}
+
+/* ------------------------------------------------------------------------- */
 /* Checkpoint-side repair of Section 6: give a fused group ONE global scale    */
 /* (the maximum of its modules' scales) and fold each module's ratio into its  */
 /* E4M3 block scales, re-rounding them:                                        */

@@ -26,7 +26,7 @@ MAX_SEGMENTS = 32
 EXPORTS = (
     "nvfp4_sf_bytes", "nvfp4_calibrate", "nvfp4_quantize_act", "nvfp4_swiglu_quantize", "nvfp4_rmsnorm_quantize",
     "nvfp4_quantize_weight",
-    "nvfp4_harmonize_scales", "nvfp4_linear", "nvfp4_linear_workspace_bytes", "nvfp4_linear_bf16",
+    "nvfp4_harmonize_scales", "nvfp4_tensor_stats", "nvfp4_linear", "nvfp4_linear_workspace_bytes", "nvfp4_linear_bf16",
     "nvfp4_linear_bf16_workspace_bytes", "nvfp4_linear_bf16_static", "nvfp4_static_status", "nvfp4_workspace_reset", "nvfp4_device_status",
     "nvfp4_set_wait_limit_ns", "nvfp4_selftest_bounded_wait", "nvfp4_launch_count", "nvfp4_set_gemm_variant", "nvfp4_gemm_variants", "nvfp4_status_string",
 )
@@ -69,6 +69,8 @@ def lib() -> ctypes.CDLL:
     L.nvfp4_quantize_weight.argtypes = [vp, i64, i64, i64, segp, i32, vp, i32, vp, vp, i32, vp]
     L.nvfp4_harmonize_scales.restype = i32
     L.nvfp4_harmonize_scales.argtypes = [vp, i64, i64, i32, segp, vp, i32, vp, vp, vp]
+    L.nvfp4_tensor_stats.restype = i32
+    L.nvfp4_tensor_stats.argtypes = [vp, i64, i64, i64, vp, vp, vp]
     L.nvfp4_linear.restype = i32
     L.nvfp4_linear.argtypes = [vp, vp, vp, i64, i64, vp, vp, i64, segp, vp, i32, vp, i64, u32, vp, sz, vp]
     L.nvfp4_linear_workspace_bytes.restype = sz
@@ -231,6 +233,15 @@ def nvfp4_harmonize_scales(w_sf: torch.Tensor, N: int, K: int, segments, g_seg: 
     _check(lib().nvfp4_harmonize_scales(_ptr(w_sf), N, K, layout, _segments(pairs), _ptr(g_seg), len(pairs),
                                         _ptr(out), _ptr(g_shared), _stream(stream)), "nvfp4_harmonize_scales")
     return out, g_shared
+
+
+def nvfp4_tensor_stats(x: torch.Tensor, g: torch.Tensor, stream=None) -> torch.Tensor:
+    """Seven float64 accumulators (see include/nvfp4.h): sums of x^2, x^4, err^2, amax, blocks, 1-hot blocks."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
+    out = torch.empty(7, dtype=torch.float64, device=x.device)
+    _check(lib().nvfp4_tensor_stats(_ptr(x), x.shape[0], x.shape[1], x.stride(0), _ptr(g), _ptr(out), _stream(stream)),
+           "nvfp4_tensor_stats")
+    return out
 
 
 def alloc_workspace(device, M: int = 0, N: int = 0, K: int = 0, nseg: int = 1, fused: bool = False) -> torch.Tensor:

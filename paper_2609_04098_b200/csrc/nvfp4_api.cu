@@ -501,6 +501,35 @@ nvfp4_status nvfp4_rmsnorm_quantize(const void* d_x, int64_t M, int64_t K, int64
                          reinterpret_cast<const uint16_t*>(d_weight), eps);
 }
 
+nvfp4_status nvfp4_tensor_stats(const void* d_x, int64_t rows, int64_t cols, int64_t ld, const float* d_g,
+                                double* d_out, void* stream) {
+    if (d_x == nullptr || d_g == nullptr || d_out == nullptr) return NVFP4_ERR_NULL;
+    if (rows < 0 || cols <= 0 || (cols % 16) != 0 || ld < cols || cols >= (1ll << 31) || rows >= (1ll << 31))
+        return NVFP4_ERR_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(d_x) & 31u) != 0 || (ld % 16) != 0 || (reinterpret_cast<uintptr_t>(d_out) & 7u) != 0)
+        return NVFP4_ERR_ALIGN;
+    DeviceInfo info;
+    nvfp4_status st = check_arch(info);
+    if (st != NVFP4_OK) return st;
+    cudaStream_t s = as_stream(stream);
+    // out[0..5] accumulators, out[6] (first 4 bytes) the running maximum as float bits
+    if (cudaMemsetAsync(d_out, 0, 7 * sizeof(double), s) != cudaSuccess) return NVFP4_ERR_CUDA;
+    const int64_t blocks16 = rows * (cols / 16);
+    if (blocks16 > 0) {
+        int64_t grid = (blocks16 + 255) / 256;
+        if (grid > info.sm_count * 8) grid = info.sm_count * 8;
+        stats_kernel<<<static_cast<int>(grid), 256, 0, s>>>(reinterpret_cast<const uint16_t*>(d_x),
+                                                            static_cast<int32_t>(rows), static_cast<int32_t>(cols), ld,
+                                                            d_g, d_out, reinterpret_cast<uint32_t*>(d_out + 6));
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        if (cudaGetLastError() != cudaSuccess) return NVFP4_ERR_CUDA;
+    }
+    stats_finalize_kernel<<<1, 1, 0, s>>>(d_out, reinterpret_cast<const uint32_t*>(d_out + 6),
+                                          static_cast<double>(blocks16));
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+}
+
 size_t nvfp4_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int nseg) {
     (void)K; (void)nseg;
     return kStatusBytes + split_area(M, N).total();

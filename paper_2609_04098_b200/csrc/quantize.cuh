@@ -299,6 +299,87 @@ quantize_kernel(const uint16_t* __restrict__ x, int32_t M, int32_t K, int64_t ld
     }
 }
 
+// ------------------------------------------------------------------ statistics
+// Columns of the paper's activation/weight statistics table at NVFP4 granularity.  One lane per
+// 16-element block; per block in binary32 (fused multiply-adds, fixed order), block results are
+// added in double: out = {sum x^2, sum x^4, sum err^2, amax (float bits in out_amax), blocks, 1-hot}.
+__global__ void __launch_bounds__(256)
+stats_kernel(const uint16_t* __restrict__ x, int32_t rows, int32_t cols, int64_t ld, const float* __restrict__ g_ptr,
+             double* __restrict__ out, uint32_t* __restrict__ out_amax) {
+    const int32_t KB = cols >> 4;
+    const int64_t total = static_cast<int64_t>(rows) * KB;
+    const float g = __ldg(g_ptr);
+    const float c1 = __fdiv_rn(1.0f, __fmul_rn(6.0f, g));
+    double t2 = 0.0, t4 = 0.0, te = 0.0, hot = 0.0;
+    float amax = 0.0f;
+    for (int64_t b = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; b < total;
+         b += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        const int64_t r = b / KB;
+        const int32_t kb = static_cast<int32_t>(b - r * KB);
+        uint32_t v[8];
+        ldg256_stream(x + r * ld + kb * 16, v);
+        float f[16];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { f[2 * i] = __uint_as_float(v[i] << 16); f[2 * i + 1] = __uint_as_float(v[i] & 0xFFFF0000u); }
+        float s2 = 0.0f, s4 = 0.0f, bmax = 0.0f;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const float q = __fmul_rn(f[i], f[i]);
+            s2 = __fmaf_rn(f[i], f[i], s2);
+            s4 = __fmaf_rn(q, q, s4);
+            bmax = fmaxf(bmax, fabsf(f[i]));
+        }
+        amax = fmaxf(amax, bmax);
+        if (__fmul_rn(__fmul_rn(bmax, bmax), 16.0f) > __fmul_rn(9.0f, s2)) hot += 1.0;
+        const uint32_t s8 = f32_to_e4m3(__fmul_rn(bmax, c1));
+        const float d = __fmul_rn(e4m3_to_f32(s8), g);
+        const float qinv = __fdiv_rn(1.0f, d);
+        float y[8];
+        float se = 0.0f;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) y[i] = __fmul_rn(f[8 * h + i], qinv);
+            const uint32_t codes = (s8 == 0u) ? 0u : f32x8_to_e2m1(y);
+            // decode the codes again (E2M1 -> fp16 is exact)
+            uint32_t h0, h1, h2, h3;
+            asm("{\n\t.reg .b8 b0, b1, b2, b3;\n\tmov.b32 {b0, b1, b2, b3}, %4;\n\t"
+                "cvt.rn.f16x2.e2m1x2 %0, b0;\n\tcvt.rn.f16x2.e2m1x2 %1, b1;\n\t"
+                "cvt.rn.f16x2.e2m1x2 %2, b2;\n\tcvt.rn.f16x2.e2m1x2 %3, b3;\n\t}\n"
+                : "=r"(h0), "=r"(h1), "=r"(h2), "=r"(h3) : "r"(codes));
+            const uint32_t hh[4] = {h0, h1, h2, h3};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float2 dq = __half22float2(*reinterpret_cast<const __half2*>(&hh[i]));
+                const float e0 = __fsub_rn(f[8 * h + 2 * i], (s8 == 0u) ? 0.0f : __fmul_rn(dq.x, d));
+                const float e1 = __fsub_rn(f[8 * h + 2 * i + 1], (s8 == 0u) ? 0.0f : __fmul_rn(dq.y, d));
+                se = __fmaf_rn(e0, e0, se);
+                se = __fmaf_rn(e1, e1, se);
+            }
+        }
+        t2 += static_cast<double>(s2); t4 += static_cast<double>(s4); te += static_cast<double>(se);
+    }
+    // warp, then device reduction
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) {
+        t2 += __shfl_xor_sync(0xffffffffu, t2, off);
+        t4 += __shfl_xor_sync(0xffffffffu, t4, off);
+        te += __shfl_xor_sync(0xffffffffu, te, off);
+        hot += __shfl_xor_sync(0xffffffffu, hot, off);
+        amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, off));
+    }
+    if ((threadIdx.x & 31) == 0) {
+        atomicAdd(out + 0, t2); atomicAdd(out + 1, t4); atomicAdd(out + 2, te); atomicAdd(out + 5, hot);
+        atomicMax(out_amax, __float_as_uint(amax));
+    }
+}
+
+// out[3] = amax, out[4] = number of blocks
+__global__ void stats_finalize_kernel(double* __restrict__ out, const uint32_t* __restrict__ amax_bits, double blocks) {
+    out[3] = static_cast<double>(__uint_as_float(*amax_bits));
+    out[4] = blocks;
+}
+
 // ------------------------------------------------------------------ scale harmonisation
 // Shared global scale for a fused group: g* = max_j g_j; every scale byte of module j becomes
 // e4m3(e4m3(s) * (g_j / g*)).  One thread handles the four scale bytes of one row and one
