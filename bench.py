@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the NVFP4 W4A4 linear-layer path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload mlp|quantize|gdn|linear]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload mlp|gdn|linear] [--tokens M]
     python bench.py --impl reference ...        # times the CPU oracle instead
 
 Default workload ("mlp"): one step = one pass of the hot path over the MLP prefill
@@ -9,8 +9,10 @@ pair of a 27B-class hybrid layer, M = 8192 tokens:
     quantize X1 [8192 x 5120] -> fused gate/up GEMM (N = 2 x 17408, two segments,
     separate global scales) -> quantize X2 [8192 x 17408] -> down GEMM (N = 5120).
 The headline value is GEMM FLOPs of the step divided by the WHOLE step time
-(quantization included).  The quantize kernel is also timed alone on the
-heavy-tailed 8192 x 5120 activation tensor and reported under "quantize".
+(quantization included).  Also reported: the GEMM's roofline fraction (events around
+each launch inside the timed region), the quantize kernel alone on the heavy-tailed
+8192 x 5120 activation tensor ("quantize"), the producer-fused quantizers, an
+end-to-end arm with host buffers ("e2e") and the CPU oracle on a sample ("cpu_baseline").
 
 Prints one JSON line (rank 0).  Multi-GPU runs are independent replicas (the path
 has no exchange step): every rank runs the same step on its own GPU.
@@ -20,7 +22,6 @@ from __future__ import annotations
 import argparse
 import json
 import os
-import subprocess
 import sys
 import threading
 import time

@@ -132,19 +132,16 @@ def _swiglu_case(M, inner, layout=nv.SF_MMA, seed=9, ld_pad=0):
     gu[:, 7] = synth.f64_to_bf16_bits(synth.bf16_bits_to_f32(gu[:, 7]).astype(np.float64) * 12.0)
     h = oracle.swiglu_bf16(gu)
     _, g = oracle.calibrate(h)
-    t = synth.to_torch_bf16(gu).to(gu_mod.DEV)
+    t = synth.to_torch_bf16(gu).to(gu.DEV)
     if ld_pad:
-        buf = torch.zeros((M, 2 * inner + ld_pad), dtype=torch.bfloat16, device=gu_mod.DEV)
+        buf = torch.zeros((M, 2 * inner + ld_pad), dtype=torch.bfloat16, device=gu.DEV)
         buf[:, :2 * inner] = t
         t = buf[:, :2 * inner]
-    codes_d, sf_d = nv.nvfp4_swiglu_quantize(t, gu_mod.dev_f32(g), layout)
+    codes_d, sf_d = nv.nvfp4_swiglu_quantize(t, gu.dev_f32(g), layout)
     torch.cuda.synchronize()
-    codes_o, sf_o, _, _ = gu_mod.oracle_quantized(h, g=g)
-    gu_mod.check_quantized(codes_d, sf_d, layout, codes_o, sf_o, inner)
+    codes_o, sf_o, _, _ = gu.oracle_quantized(h, g=g)
+    gu.check_quantized(codes_d, sf_d, layout, codes_o, sf_o, inner)
     return t, g, codes_d, sf_d
-
-
-from tests import gpu_util as gu_mod  # noqa: E402  (alias: `gu` above is the helper module too)
 
 
 @pytest.mark.parametrize("M,inner", [(1, 16), (5, 48), (128, 512), (130, 1040), (300, 17408 // 4)])
@@ -156,9 +153,9 @@ def test_swiglu_quantize_matches_oracle_composition(M, inner, layout):
 def test_swiglu_quantize_strided_and_equal_to_unfused_path():
     t, g, codes_d, sf_d = _swiglu_case(96, 2048, ld_pad=64)
     # the same result as materialising h in bf16 and calling nvfp4_quantize_act on it
-    gu_host = gu_mod.host_bits(t.contiguous())
-    h = gu_mod.dev_bf16(oracle.swiglu_bf16(gu_host))
-    c2, s2 = nv.nvfp4_quantize_act(h, gu_mod.dev_f32(g))
+    gu_host = gu.host_bits(t.contiguous())
+    h = gu.dev_bf16(oracle.swiglu_bf16(gu_host))
+    c2, s2 = nv.nvfp4_quantize_act(h, gu.dev_f32(g))
     torch.cuda.synchronize()
     assert torch.equal(c2, codes_d) and torch.equal(s2, sf_d)
 
@@ -171,10 +168,10 @@ def test_swiglu_extreme_gates():
     gu = synth.f64_to_bf16_bits(vals).reshape(M, 2 * inner)
     h = oracle.swiglu_bf16(gu)
     _, g = oracle.calibrate(h)
-    codes_d, sf_d = nv.nvfp4_swiglu_quantize(gu_mod.dev_bf16(gu), gu_mod.dev_f32(g))
+    codes_d, sf_d = nv.nvfp4_swiglu_quantize(gu.dev_bf16(gu), gu.dev_f32(g))
     torch.cuda.synchronize()
-    codes_o, sf_o, _, _ = gu_mod.oracle_quantized(h, g=g)
-    gu_mod.check_quantized(codes_d, sf_d, nv.SF_MMA, codes_o, sf_o, inner)
+    codes_o, sf_o, _, _ = gu.oracle_quantized(h, g=g)
+    gu.check_quantized(codes_d, sf_d, nv.SF_MMA, codes_o, sf_o, inner)
 
 
 # ---- producer fusion: RMSNorm(x) * w -> quantize in one pass ----------------------------------
@@ -183,15 +180,15 @@ def _rmsnorm_case(M, K, layout=nv.SF_MMA, seed=12, eps=1e-6, ld_pad=0):
     w = synth.f64_to_bf16_bits(1.0 + 0.25 * np.cos(0.37 * np.arange(K)))
     y = oracle.rmsnorm_bf16(x, w, eps)
     _, g = oracle.calibrate(y)
-    t = gu_mod.dev_bf16(x)
+    t = gu.dev_bf16(x)
     if ld_pad:
-        buf = torch.zeros((M, K + ld_pad), dtype=torch.bfloat16, device=gu_mod.DEV)
+        buf = torch.zeros((M, K + ld_pad), dtype=torch.bfloat16, device=gu.DEV)
         buf[:, :K] = t
         t = buf[:, :K]
-    codes_d, sf_d = nv.nvfp4_rmsnorm_quantize(t, gu_mod.dev_bf16(w), eps, gu_mod.dev_f32(g), layout)
+    codes_d, sf_d = nv.nvfp4_rmsnorm_quantize(t, gu.dev_bf16(w), eps, gu.dev_f32(g), layout)
     torch.cuda.synchronize()
-    codes_o, sf_o, _, _ = gu_mod.oracle_quantized(y, g=g)
-    gu_mod.check_quantized(codes_d, sf_d, layout, codes_o, sf_o, K)
+    codes_o, sf_o, _, _ = gu.oracle_quantized(y, g=g)
+    gu.check_quantized(codes_d, sf_d, layout, codes_o, sf_o, K)
 
 
 @pytest.mark.parametrize("M,K", [(1, 16), (3, 528), (130, 5120), (64, 17408), (257, 1040)])
