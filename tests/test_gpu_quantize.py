@@ -127,12 +127,12 @@ def test_gdn_weight_full_size():
 # ---- producer fusion: silu(gate) * up -> quantize in one pass -------------------------------
 def _swiglu_case(M, inner, layout=nv.SF_MMA, seed=9, ld_pad=0):
     segs = synth.make_segments((("gate", M, 1.0),))
-    gu = synth.weights(seed, 60, segs, 2 * inner)                 # bf16 [M, 2*inner] ~ N(0, 1): gate | up
+    gate_up = synth.weights(seed, 60, segs, 2 * inner)                 # bf16 [M, 2*inner] ~ N(0, 1): gate | up
     # a few hot entries, as after a projection of outlier channels
-    gu[:, 7] = synth.f64_to_bf16_bits(synth.bf16_bits_to_f32(gu[:, 7]).astype(np.float64) * 12.0)
-    h = oracle.swiglu_bf16(gu)
+    gate_up[:, 7] = synth.f64_to_bf16_bits(synth.bf16_bits_to_f32(gate_up[:, 7]).astype(np.float64) * 12.0)
+    h = oracle.swiglu_bf16(gate_up)
     _, g = oracle.calibrate(h)
-    t = synth.to_torch_bf16(gu).to(gu.DEV)
+    t = synth.to_torch_bf16(gate_up).to(gu.DEV)
     if ld_pad:
         buf = torch.zeros((M, 2 * inner + ld_pad), dtype=torch.bfloat16, device=gu.DEV)
         buf[:, :2 * inner] = t
@@ -165,10 +165,10 @@ def test_swiglu_extreme_gates():
     vals = np.zeros((M, 2 * inner))
     vals[:, :inner] = np.linspace(-120, 120, inner)[None, :] * np.array([1.0, 0.5, 0.01, -1.0])[:, None]
     vals[:, inner:] = np.array([1.0, -3.0, 250.0, 0.125])[:, None]
-    gu = synth.f64_to_bf16_bits(vals).reshape(M, 2 * inner)
-    h = oracle.swiglu_bf16(gu)
+    gate_up = synth.f64_to_bf16_bits(vals).reshape(M, 2 * inner)
+    h = oracle.swiglu_bf16(gate_up)
     _, g = oracle.calibrate(h)
-    codes_d, sf_d = nv.nvfp4_swiglu_quantize(gu.dev_bf16(gu), gu.dev_f32(g))
+    codes_d, sf_d = nv.nvfp4_swiglu_quantize(gu.dev_bf16(gate_up), gu.dev_f32(g))
     torch.cuda.synchronize()
     codes_o, sf_o, _, _ = gu.oracle_quantized(h, g=g)
     gu.check_quantized(codes_d, sf_d, nv.SF_MMA, codes_o, sf_o, inner)
