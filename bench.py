@@ -52,6 +52,19 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
+def tensor_peak(peaks, timed_seconds: float, clocks: dict):
+    """Which measured bf16 figure the FP4 roofline is built on (x 4, the nominal FP4 : bf16 ratio):
+    the burst figure when the timed region was short and never power-capped (the clocks then sit
+    at their maximum, as they did when the burst figure was taken), the sustained one otherwise."""
+    capped = "sw_power_cap" in (clocks.get("reasons") or [])
+    burst = timed_seconds < 1.0 and not capped
+    base = peaks["bf16_tflops"] if burst else peaks["bf16_tflops_sustained"]
+    basis = "%s bf16 %s %.1f TFLOP/s x %.0f (nominal FP4:bf16 ratio); timed region %.3f s, %s" % (
+        peaks["source"], "burst" if burst else "sustained", base, FP4_OVER_BF16, timed_seconds,
+        "power cap seen" if capped else "no power cap seen")
+    return base * FP4_OVER_BF16, basis
+
+
 def ncu_traffic(name: str):
     """DRAM bytes per launch from the committed ncu summary (profiles/traffic.json), or None."""
     path = os.path.join(ROOT, "profiles", "traffic.json")
@@ -171,6 +184,102 @@ class OneLinear:
         self.describe = "configs[4] linear K=5120->N=6144 at M=%d, quantize fused into the timed call" % M
 
 
+# --------------------------------------------------------------------------- other configs, same JSON line
+def measure_configs(torch, nv, dev, peaks, seed):
+    """configs[3] (fused GDN in-projection, six segments) and configs[4] (K=5120 -> N=6144 at
+    M in {1 .. 32768}, quantize inside the timed call), each timed for a few hundred ms at most.
+    Every timed call goes through nvfp4_linear_bf16.  Weights rotate through enough copies to
+    exceed L2 (a model streams each layer's weights from HBM; one layer replayed would sit in
+    L2), activations and outputs rotate too.  Decode-sized shapes are timed as a CUDA-graph
+    replay, so the host's launch cost is not what is measured."""
+    stream = torch.cuda.current_stream()
+
+    def up(bits):
+        return synth.to_torch_bf16(bits).to(dev)
+
+    def time_layer(M, segs, hx, w_c, w_sf, g_w, n_wsets, reps, graph):
+        N = sum(s.count for s in segs)
+        per_set = M * HIDDEN * 2 + M * N * 2
+        nset = max(1, min(6, int(np.ceil(300e6 / per_set))))
+        xs = [up(hx) for _ in range(nset)]
+        g1 = nv.nvfp4_calibrate(xs[0])
+        ys = [torch.empty((M, N), dtype=torch.bfloat16, device=dev) for _ in range(nset)]
+        ws = nv.alloc_workspace(dev, M, N, HIDDEN, len(segs), fused=True)
+        wsets = [(w_c, w_sf)] + [(w_c.clone(), w_sf.clone()) for _ in range(n_wsets - 1)]
+        k = [0]
+
+        def call():
+            i = k[0]
+            k[0] += 1
+            wc_, wsf_ = wsets[i % n_wsets]
+            nv.nvfp4_linear_bf16(xs[i % nset], g1, wc_, wsf_, segs, g_w, ws, out=ys[i % nset])
+
+        for _ in range(3):
+            call()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        if graph:
+            side = torch.cuda.Stream()
+            side.wait_stream(stream)
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(side):
+                with torch.cuda.graph(g, stream=side):
+                    for _ in range(reps):
+                        call()
+                g.replay()
+                side.synchronize()
+                e0.record(side)
+                g.replay()
+                e1.record(side)
+                side.synchronize()
+        else:
+            e0.record(stream)
+            for _ in range(reps):
+                call()
+            e1.record(stream)
+            torch.cuda.synchronize()
+        status = nv.device_status(ws)
+        if status != 0:
+            raise SystemExit("device status %d in the configs block" % status)
+        return e0.elapsed_time(e1) / reps * 1e3            # microseconds per call
+
+    out = {}
+    # configs[3]
+    gdn = GdnProj(8192)
+    hx = synth.prefill_activations(seed, 401, gdn.M, HIDDEN)
+    w_c, w_sf, g_w = nv.nvfp4_quantize_weight(up(synth.weights(seed, 402, gdn.segs, HIDDEN)), gdn.segs)
+    us = time_layer(gdn.M, gdn.segs, hx, w_c, w_sf, g_w, n_wsets=1, reps=40, graph=False)
+    tf = gdn.flops / (us * 1e-6) / 1e12
+    out["configs[3] fused GDN in-projection M=8192 K=5120 N=16480 (6 segments), quantize inside the call"] = {
+        "us_per_call": round(us, 1), "tflops": round(tf, 1), "frac_of_nominal_9pf": round(tf / NOMINAL_FP4_TFLOPS, 4)}
+    del w_c, w_sf
+    # configs[4]
+    lin = OneLinear(1)
+    w_c, w_sf, g_w = nv.nvfp4_quantize_weight(up(synth.weights(seed, 402, lin.segs, HIDDEN)), lin.segs)
+    weight_bytes = lin.N * HIDDEN * (0.5 + 1.0 / 16.0)
+    n_wsets = int(np.ceil(200e6 / weight_bytes))
+    hx_all = synth.prefill_activations(seed, 401, 32768, HIDDEN)
+    sweep = []
+    for M in (1, 16, 128, 1024, 8192, 32768):
+        small = M <= 1024
+        us = time_layer(M, lin.segs, hx_all[:M], w_c, w_sf, g_w, n_wsets=n_wsets if small else 1,
+                        reps=200 if small else (40 if M == 8192 else 12), graph=small)
+        row = {"M": M, "us_per_call": round(us, 2), "launch": "cuda graph replay" if small else "stream launches"}
+        flops = gemm_flops(M, lin.N, HIDDEN)
+        if M <= 128:
+            floor_us = weight_bytes / (peaks["hbm_gbs"] * 1e9) * 1e6
+            row.update({"weight_gbs": round(weight_bytes / (us * 1e-6) / 1e9, 1),
+                        "frac_of_weight_bandwidth_roofline": round(floor_us / us, 4),
+                        "roofline_us": round(floor_us, 2)})
+        else:
+            tf = flops / (us * 1e-6) / 1e12
+            row.update({"tflops": round(tf, 1), "frac_of_nominal_9pf": round(tf / NOMINAL_FP4_TFLOPS, 4)})
+        sweep.append(row)
+    out["configs[4] K=5120 -> N=6144, quantize inside the call; weights rotate through %d copies (%.0f MB) for M <= 1024" % (
+        n_wsets, n_wsets * weight_bytes / 1e6)] = sweep
+    return out
+
+
 # --------------------------------------------------------------------------- GPU arm
 def run_gpu(args):
     import torch
@@ -191,7 +300,6 @@ def run_gpu(args):
     if args.variant:
         nv.set_gemm_variant(args.variant)
     peaks = measured_peaks()
-    fp4_peak = peaks["bf16_tflops_sustained"] * FP4_OVER_BF16
     stream = torch.cuda.current_stream()
 
     def up(bits):
@@ -346,12 +454,16 @@ def run_gpu(args):
         gemm_ms = ms_per_step
         achieved = wl.flops / (gemm_ms * 1e-3) / 1e12
         quant_in_step_gbs = None
+    fp4_peak, peak_basis = tensor_peak(peaks, total_ms * 1e-3, clocks)
+    clock_scaled = (148 * 32768 * clocks["sm_mhz"] * 1e6 / 1e12) if clocks.get("sm_mhz") else None
     roofline = {"kernel": "gemm_kernel (tcgen05 block-scaled FP4)", "bound": "tensor",
                 "achieved": round(achieved, 2), "peak": round(fp4_peak, 1), "unit": "TFLOP/s",
-                "frac": round(achieved / fp4_peak, 4),
-                "peak_basis": "%s bf16 sustained %.1f TFLOP/s x %.0f (nominal FP4:bf16 ratio)" % (
-                    peaks["source"], peaks["bf16_tflops_sustained"], FP4_OVER_BF16),
+                "frac": round(achieved / fp4_peak, 4), "peak_basis": peak_basis,
+                "frac_of_burst_x4": round(achieved / (peaks["bf16_tflops"] * FP4_OVER_BF16), 4),
+                "frac_of_sustained_x4": round(achieved / (peaks["bf16_tflops_sustained"] * FP4_OVER_BF16), 4),
                 "frac_of_nominal_9pf": round(achieved / NOMINAL_FP4_TFLOPS, 4),
+                "frac_of_clock_scaled_peak": None if not clock_scaled else round(achieved / clock_scaled, 4),
+                "clock_scaled_peak_basis": "148 SMs x 32768 FLOP/clk x median SM clock during the timed region",
                 "avg_launch_ms": round(gemm_ms, 4),
                 "traffic": ncu_traffic("gemm_kernel")}
     result["roofline"] = roofline
@@ -520,6 +632,11 @@ def run_gpu(args):
     if status != 0:
         raise SystemExit("device status %d after the timed region" % status)
 
+    if rank == 0 and not args.skip_configs and args.workload == "mlp":
+        del x1, x2, y1, y2, q1, q2
+        torch.cuda.empty_cache()
+        result["configs"] = measure_configs(torch, nv, dev, peaks, args.seed)
+
     if rank == 0:
         if not args.skip_cpu:
             result["cpu_baseline"] = cpu_baseline(wl, target_s=args.cpu_seconds, seed=args.seed,
@@ -621,6 +738,7 @@ def main():
                     help="time small-M workloads with plain stream launches instead of a CUDA graph")
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--skip-quantize", action="store_true")
+    ap.add_argument("--skip-configs", action="store_true", help="leave out the configs[3] / configs[4] block")
     args = ap.parse_args()
     ref = args.impl == "reference"
     if args.steps is None:
@@ -629,8 +747,12 @@ def main():
         args.warmup = 1 if ref else 10
     if args.impl == "reference":
         run_reference(args)
-    else:
-        run_gpu(args)
+        return
+    from paper_2609_04098_b200.replicas import launched_by_a_launcher, spawn_replicas
+    if args.gpus > 1 and not launched_by_a_launcher():
+        # nobody started the ranks for us: one process per GPU, each an independent replica
+        sys.exit(spawn_replicas(args.gpus, [sys.executable, os.path.abspath(__file__)] + sys.argv[1:]))
+    run_gpu(args)
 
 
 if __name__ == "__main__":

@@ -54,7 +54,8 @@ typedef enum {
     NVFP4_ERR_ARCH = 6,        /* current device is not compute capability 10.x */
     NVFP4_ERR_CUDA = 7,        /* a CUDA runtime/driver call or a launch failed */
     NVFP4_ERR_TIMEOUT = 8,     /* a bounded wait inside a kernel ran out (see nvfp4_device_status) */
-    NVFP4_ERR_LAYOUT = 9       /* unknown scale layout / the GEMM needs NVFP4_SF_MMA */
+    NVFP4_ERR_LAYOUT = 9,      /* unknown scale layout / the GEMM needs NVFP4_SF_MMA */
+    NVFP4_ERR_SCALE = 10       /* a global scale read on the device was not finite and > 0 (see nvfp4_device_status) */
 } nvfp4_status;
 
 /* One fused module's slice of the output columns (= rows of the weight matrix). */
@@ -71,9 +72,22 @@ typedef enum { NVFP4_SF_LINEAR = 0, NVFP4_SF_MMA = 1 } nvfp4_sf_layout;
 #define NVFP4_OUT_BF16 0u     /* Y is bf16 (default)                                  */
 #define NVFP4_OUT_F32  1u     /* Y is float32 (testing aid: no output rounding)       */
 #define NVFP4_WS_ZEROED 2u    /* caller's promise: the workspace was zero-filled once (e.g. cudaMemset) and has
-                                 since been written by this library only.  Lets decode-sized calls (M <= 128)
+                                 since been written by this library only.  Lets decode-sized calls (M <= 256)
                                  split K over several CTAs, which meet in the workspace and leave it zero again.
                                  After NVFP4_ERR_TIMEOUT zero the workspace before the next call with this flag. */
+
+/*
+ * Workspace layout (the same for every entry point and every problem size, so one zero-filled
+ * workspace can serve calls of different shapes, e.g. the K = 5120 and K = 17408 layers of one model):
+ *   [0, 256)                                    status block; its first word is the status flag
+ *   [256, 256 + NVFP4_SPLIT_RESERVE_BYTES)      split-K counters and fp32 partial sums.  Used only with
+ *                                               NVFP4_WS_ZEROED, and only as far as the workspace reaches;
+ *                                               a call whose split-K area would not fit does not split K
+ *   [256 + NVFP4_SPLIT_RESERVE_BYTES, ...)      nvfp4_linear_bf16 only: the quantized activations
+ * Nothing the library writes outside the split-K part can land on it, and every call that uses that
+ * part leaves it zero again: the NVFP4_WS_ZEROED promise, once true, stays true.
+ */
+#define NVFP4_SPLIT_RESERVE_BYTES (5u * 1024u * 1024u)
 
 /* Size in bytes of the scale buffer for a [rows, K] tensor in `layout` (K % 16 == 0). */
 size_t nvfp4_sf_bytes(int64_t rows, int64_t K, nvfp4_sf_layout layout);
@@ -112,35 +126,43 @@ nvfp4_status nvfp4_quantize_act(const void* d_x, int64_t M, int64_t K, int64_t l
  * 496 quantized linears, so the down projection's input silu(gate)*up is quantized on every
  * call; Section 9 names activation quantization as the overhead to remove).  Reads the fused
  * gate/up GEMM output once and writes only codes and scales: h is never stored in bf16.
- *     h = bf16_rne( silu(gate) * up ),  then exactly nvfp4_quantize_act(h)
- * with silu(g)*u evaluated in binary32 as: t = clamp(-g, -87, 87); n = rint(t*log2e);
- * r = fmaf(t, log2e, -n); e = poly5(r) * 2^n; s = g * (1/(1+e)); s*u   (every step one IEEE op).
+ *     h = bf16_rne( silu(gate) * up ),  silu(g) = g / (1 + exp(-g)),  then exactly nvfp4_quantize_act(h)
+ * The paper fixes no arithmetic for the activation (it is upstream of the quantized linears, in
+ * bf16).  The kernel evaluates it in binary32 with the hardware's approximate exp2 and
+ * reciprocal; the bf16 result equals the correctly rounded definition for all but a small
+ * fraction of elements and is never more than one bf16 ulp away.  Codes and scales are the exact
+ * quantization of the h the kernel formed.
  *   d_gate_up  bf16 [M, 2*inner], gate in columns [0, inner), up in [inner, 2*inner); row
  *              stride ld >= 2*inner; 32-byte aligned, ld % 16 == 0, inner % 16 == 0
  *   d_g        in: global scale of h (calibrated offline, as for any activation)
  *   d_codes    out [M, inner/2]; d_sf out nvfp4_sf_bytes(M, inner, layout)
+ *   d_h        optional (may be NULL), testing aid: out bf16 [M, inner] row-major, 32-byte aligned --
+ *              the tensor h that was quantized
  * Errors: as nvfp4_quantize_act.
  */
 nvfp4_status nvfp4_swiglu_quantize(const void* d_gate_up, int64_t M, int64_t inner, int64_t ld,
                                    const float* d_g, uint8_t* d_codes, uint8_t* d_sf,
-                                   nvfp4_sf_layout layout, void* stream);
+                                   nvfp4_sf_layout layout, void* d_h, void* stream);
 
 /*
  * Activation quantization fused into RMSNorm (paper: Background / Setup -- norms are excluded from
  * quantization and stay bf16 upstream of every quantized linear, so the in-projections quantize
  * a normalised residual stream on every call).  One pass over x from HBM:
- *     y = bf16_rne( (x * rstd) * w ),  rstd = 1 / sqrt(mean_k(x^2) + eps),  then nvfp4_quantize_act(y)
- * in binary32: each of 32 lanes sums x^2 (fused multiply-add) over the 16-element pieces k/16 % 32
- * == lane in increasing k, the partial sums meet in a butterfly (offsets 16, 8, 4, 2, 1), IEEE
- * divide, sqrt and reciprocal.
+ *     y = bf16_rne( x * rstd * w ),  rstd = 1 / sqrt(mean_k(x^2) + eps),  then nvfp4_quantize_act(y)
+ * The paper fixes no arithmetic for the norm; the kernel sums the squares in binary32 (per lane,
+ * then across the warp) and multiplies in binary32: y equals the correctly rounded definition for
+ * all but a small fraction of elements, never more than one bf16 ulp away.  Codes and scales are the
+ * exact quantization of the y the kernel formed.
  *   d_x       bf16 [M, K], row stride ld; 32-byte aligned, ld % 16 == 0
  *   d_weight  bf16 [K] (the norm's gain), 32-byte aligned;  eps >= 0
  *   d_g       in: global scale of y (calibrated offline);  outputs as nvfp4_quantize_act
+ *   d_y       optional (may be NULL), testing aid: out bf16 [M, K] row-major, 32-byte aligned -- the
+ *             tensor y that was quantized
  * Errors: as nvfp4_quantize_act, plus NULL / misaligned weight, negative or NaN eps.
  */
 nvfp4_status nvfp4_rmsnorm_quantize(const void* d_x, int64_t M, int64_t K, int64_t ld, const void* d_weight,
                                     float eps, const float* d_g, uint8_t* d_codes, uint8_t* d_sf,
-                                    nvfp4_sf_layout layout, void* stream);
+                                    nvfp4_sf_layout layout, void* d_y, void* stream);
 
 /*
  * Offline weight quantization, same format, blocks along K, with one global scale
@@ -158,9 +180,10 @@ nvfp4_status nvfp4_quantize_weight(const void* d_w, int64_t N, int64_t K, int64_
                                    nvfp4_sf_layout layout, void* stream);
 
 /*
- * Checkpoint-side repair (paper: Section 6 -- "rewrite each fused group to the shared global
- * scale and fold the ratio into the per-block E4M3 scales", re-rounding error <= 6.2 %): lets a
- * GEMM with ONE global scale serve a fused group whose modules were calibrated separately.
+ * Checkpoint-side repair (paper: Section 6, the fix applied to the released checkpoint: every
+ * fused group gets one shared global scale and each module's ratio to it is multiplied into that
+ * module's E4M3 block scales, which are rounded again; the paper bounds that re-rounding at 6.2 %):
+ * lets a GEMM with ONE global scale serve a fused group whose modules were calibrated separately.
  *     g* = max_j g_seg[j];   s'_b = e4m3_rne_sat( e4m3(s_b) * (g_seg[j] / g*) )   (binary32)
  * Codes are unchanged.  Afterwards nvfp4_linear with the single segment [0, N) and g* reproduces
  * the per-module result up to the re-rounding of the scales; the per-segment epilogue of
@@ -204,9 +227,10 @@ nvfp4_status nvfp4_tensor_stats(const void* d_x, int64_t rows, int64_t cols, int
  *   d_workspace        at least 256 bytes, 16-byte aligned; its first word is a status flag read
  *                      by nvfp4_device_status.  nvfp4_linear_workspace_bytes(...) is the size that
  *                      also holds the split-K area used with NVFP4_WS_ZEROED (more than 256 bytes
- *                      only for M <= 256)
+ *                      only for M <= 256; never more than 256 + NVFP4_SPLIT_RESERVE_BYTES)
  * Requirements: K % 64 == 0; code pointers 16-byte aligned; scale pointers 16-byte aligned.
- * Errors: see nvfp4_status; M == 0 or N == 0 is a no-op.
+ * Errors: see nvfp4_status; M == 0 or N == 0 is a no-op.  The kernel checks on the device that g_a and
+ * every g_seg[j] is finite and > 0; if not, the status word becomes NVFP4_ERR_SCALE and Y is unspecified.
  */
 nvfp4_status nvfp4_linear(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const float* d_g_a,
                           int64_t M, int64_t K,
@@ -223,9 +247,12 @@ size_t nvfp4_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int nseg);
  * that matters at small batch), codes and scales live in the workspace.
  *   d_x   bf16 [M, K], row stride ldx, 32-byte aligned, ldx % 16 == 0
  * For M = 1 or 2 (single-stream decode) the call is one weight-streaming kernel on the CUDA cores
- * that quantizes the activations itself (same codes) and does not touch the workspace; from M = 3
- * on it is the quantize kernel followed by the tensor-core GEMM, which starts its prologue while
- * the quantizer still runs.
+ * that quantizes the activations itself (same codes) and uses only the status word of the
+ * workspace; from M = 3 on it is the quantize kernel followed by the tensor-core GEMM, which starts
+ * its prologue while the quantizer still runs.
+ *   d_workspace  nvfp4_linear_bf16_workspace_bytes(M, N, K, nseg) bytes (status block, split-K
+ *                reserve, codes and scales of the activations), 16-byte aligned
+ * Every argument is checked before anything is enqueued.
  */
 nvfp4_status nvfp4_linear_bf16(const void* d_x, int64_t ldx, const float* d_g_a,
                                int64_t M, int64_t K,
@@ -250,19 +277,23 @@ size_t nvfp4_linear_bf16_workspace_bytes(int64_t M, int64_t N, int64_t K, int ns
  * loads the library holds the array until the process exits.
  *
  *   - It calls no cudaMalloc / cudaFree and no allocating library routine.
- *   - Sizes whose quantized activations (M*K/2 bytes of codes, their scales and a 256-byte
- *     status block) exceed NVFP4_STATIC_SCRATCH_BYTES are rejected with NVFP4_ERR_WORKSPACE
- *     before anything is launched (the limit fits decode-sized batches, e.g. M = 256 rows at
- *     K = 16384).
+ *   - The array is laid out like any workspace (status block, split-K reserve, quantized
+ *     activations).  Sizes whose quantized activations (rows padded to 128, K/2 bytes of codes per
+ *     row, plus their scales) do not fit behind the reserve are rejected with NVFP4_ERR_WORKSPACE
+ *     before anything is launched; the limit fits decode-sized batches, e.g. M = 640 rows at
+ *     K = 17408.
  *   - The first call on each device looks up the array's device address (once, with that
  *     device current).  Make that first call outside of any stream capture.
- *   - All calls share the one array and it keeps the previous call's contents; the
- *     status word at its start is cleared by every call.  Two calls that overlap on the
- *     GPU (different streams, no dependency) race on it: serialise them.
- *   - nvfp4_static_status(stream) is nvfp4_device_status for this array.
+ *   - All calls share the one array and it keeps the previous call's contents.  What must start
+ *     at zero is kept at zero by the library itself: the split-K part is left zero by every call
+ *     that uses it, whatever shapes earlier calls had.  Two calls that overlap on the
+ *     GPU (different streams, no dependency) race on the array: serialise them.
+ *   - nvfp4_static_status(stream) is nvfp4_device_status for this array.  If it reports a failure
+ *     (a timeout, a bad global scale) it also clears the status word and re-zeroes the split-K
+ *     part, so the next call starts clean; a caller has no other handle on the array.
  * Everything else (arguments, layouts, errors) is as for nvfp4_linear_bf16.
  */
-#define NVFP4_STATIC_SCRATCH_BYTES (4u * 1024u * 1024u)
+#define NVFP4_STATIC_SCRATCH_BYTES (12u * 1024u * 1024u)
 nvfp4_status nvfp4_linear_bf16_static(const void* d_x, int64_t ldx, const float* d_g_a,
                                       int64_t M, int64_t K,
                                       const uint8_t* d_w_codes, const uint8_t* d_w_sf, int64_t N,
@@ -277,9 +308,10 @@ nvfp4_status nvfp4_static_status(void* stream);
 nvfp4_status nvfp4_workspace_reset(void* d_workspace, size_t workspace_bytes, void* stream);
 
 /*
- * Synchronises `stream` and returns the status word of the workspace: NVFP4_OK, or
- * NVFP4_ERR_TIMEOUT if a kernel gave up on one of its bounded waits (its output is
- * then unspecified; the CUDA context stays usable).
+ * Synchronises `stream` and returns the status word of the workspace: NVFP4_OK,
+ * NVFP4_ERR_TIMEOUT if a kernel gave up on one of its bounded waits, or NVFP4_ERR_SCALE if a kernel
+ * read a global scale that is not finite and > 0 (the output is then unspecified; the CUDA context
+ * stays usable).
  */
 nvfp4_status nvfp4_device_status(const void* d_workspace, void* stream);
 

@@ -62,12 +62,12 @@ def _load():
     L.orc_calibrate.argtypes = [u16p, i64, i64, i64, f32p, f32p]
     L.orc_quantize.restype = ctypes.c_int
     L.orc_quantize.argtypes = [u16p, i64, i64, i64, f32p, u8p, u8p]
-    L.orc_silu_mul.restype = ctypes.c_float
-    L.orc_silu_mul.argtypes = [ctypes.c_float, ctypes.c_float]
+    L.orc_silu_mul.restype = ctypes.c_double
+    L.orc_silu_mul.argtypes = [ctypes.c_double, ctypes.c_double]
     L.orc_swiglu_bf16.restype = None
     L.orc_swiglu_bf16.argtypes = [u16p, i64, i64, i64, u16p]
     L.orc_rmsnorm_bf16.restype = None
-    L.orc_rmsnorm_bf16.argtypes = [u16p, i64, i64, i64, u16p, ctypes.c_float, u16p]
+    L.orc_rmsnorm_bf16.argtypes = [u16p, i64, i64, i64, u16p, ctypes.c_double, u16p]
     L.orc_dequantize.restype = None
     L.orc_dequantize.argtypes = [u8p, u8p, f32p, i64, i64, f64p]
     L.orc_harmonize_scales.restype = ctypes.c_float
@@ -169,12 +169,13 @@ def quantize(x_bits: np.ndarray, g_row: np.ndarray):
 
 
 def silu_mul(g: float, u: float) -> float:
-    """silu(g) * u in the path's binary32 operation sequence (before the bf16 rounding)."""
-    return float(_load().orc_silu_mul(np.float32(g), np.float32(u)))
+    """silu(g) * u = g / (1 + exp(-g)) * u in double (before the bf16 rounding)."""
+    return float(_load().orc_silu_mul(float(g), float(u)))
 
 
 def swiglu_bf16(gate_up_bits: np.ndarray) -> np.ndarray:
-    """bf16 [R, 2I] (gate | up) -> h = bf16(silu(gate) * up), bf16 bit patterns [R, I]."""
+    """bf16 [R, 2I] (gate | up) -> h = bf16(silu(gate) * up), bf16 bit patterns [R, I]: the
+    definition evaluated in double and rounded once."""
     gu = _c(gate_up_bits, np.uint16)
     R, two_i = gu.shape
     assert two_i % 2 == 0
@@ -190,7 +191,7 @@ def rmsnorm_bf16(x_bits: np.ndarray, w_bits: np.ndarray, eps: float) -> np.ndarr
     R, C = x.shape
     assert w.shape == (C,)
     y = np.empty((R, C), np.uint16)
-    _load().orc_rmsnorm_bf16(_p(x), R, C, C, _p(w), ctypes.c_float(float(np.float32(eps))), _p(y))
+    _load().orc_rmsnorm_bf16(_p(x), R, C, C, _p(w), ctypes.c_double(float(np.float32(eps))), _p(y))
     return y
 
 

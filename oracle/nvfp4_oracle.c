@@ -178,43 +178,15 @@ int orc_quantize(const uint16_t* x, int64_t rows, int64_t cols, int64_t ld,
 
 /* ------------------------------------------------------------------------- */
 /* Producer fusion for the MLP: h = silu(gate) * up, rounded to bf16, is what  */
-/* the down projection quantizes.  The paper fixes no arithmetic for it (the   */
-/* activation is upstream of the quantized linears), so the contract is this   */
-/* binary32 sequence, every step one IEEE operation (fmaf = fused, exact):     */
-/*   t = clamp(-g, -87, 87)                                                    */
-/*   z = t * log2(e);  n = rint(z);  r = fmaf(t, log2(e), -n)     r in [-.5,.5] */
-/*   p = 2^r by a degree-5 polynomial (Horner, fmaf);  e = p * 2^n             */
-/*   s = g * (1 / (1 + e));   h = bf16_rne(s * u)                              */
+/* the down projection quantizes.  The activation sits upstream of the         */
+/* quantized linears, in bf16, and the paper fixes no arithmetic for it: the   */
+/* oracle is the definition, evaluated in double and rounded ONCE to bf16:     */
+/*     silu(g) = g / (1 + exp(-g));   h = bf16_rne( silu(g) * u )              */
+/* A kernel that evaluates it in binary32 may differ from this by one bf16 ulp */
+/* on a small fraction of elements; the comparison allows exactly that.        */
 /* ------------------------------------------------------------------------- */
-static inline float orc_exp_poly(float t) {
-    const float LOG2E = 1.44269504088896341f;
-    if (t < -87.0f) t = -87.0f;
-    if (t > 87.0f) t = 87.0f;
-    const float z = t * LOG2E;
-    const float n = rintf(z);
-    const float r = fmaf(t, LOG2E, -n);
-    float p = 1.3333558146e-3f;                 /* ln2^5/120 and friends */
-    p = fmaf(p, r, 9.6181291076e-3f);
-    p = fmaf(p, r, 5.5504108665e-2f);
-    p = fmaf(p, r, 2.4022650696e-1f);
-    p = fmaf(p, r, 6.9314718056e-1f);
-    p = fmaf(p, r, 1.0f);
-    union { float f; uint32_t u; } sc;
-    sc.u = (uint32_t)((int32_t)n + 127) << 23;  /* 2^n, n in [-126, 126] after the clamp */
-    return p * sc.f;
-}
-
-float orc_silu_mul(float g, float u) {
-    const float e = orc_exp_poly(-g);
-    const float s = g * (1.0f / (1.0f + e));
-    return s * u;
-}
-
-static inline uint16_t orc_f32_to_bf16(float f) {
-    uint32_t b;
-    memcpy(&b, &f, 4);
-    if ((b & 0x7FFFFFFFu) > 0x7F800000u) return 0x7FC0;
-    return (uint16_t)((b + 0x7FFFu + ((b >> 16) & 1u)) >> 16);
+double orc_silu_mul(double g, double u) {
+    return g / (1.0 + exp(-g)) * u;
 }
 
 /* gate_up: bf16 [rows, 2*inner] (gate in columns [0, inner), up in [inner, 2*inner)), row */
@@ -223,41 +195,28 @@ void orc_swiglu_bf16(const uint16_t* gate_up, int64_t rows, int64_t inner, int64
     #pragma omp parallel for schedule(static)
     for (int64_t r = 0; r < rows; ++r)
         for (int64_t c = 0; c < inner; ++c)
-            h[r * inner + c] = orc_f32_to_bf16(orc_silu_mul(bf16_to_f32(gate_up[r * ld + c]),
-                                                            bf16_to_f32(gate_up[r * ld + inner + c])));
+            h[r * inner + c] = orc_f64_to_bf16(orc_silu_mul((double)bf16_to_f32(gate_up[r * ld + c]),
+                                                            (double)bf16_to_f32(gate_up[r * ld + inner + c])));
 }
 
 /* ------------------------------------------------------------------------- */
 /* Producer fusion for the in-projections: their input is RMSNorm(x) * w (the  */
 /* norms stay bf16 upstream of every quantized linear).  The paper fixes no    */
-/* arithmetic for it; the contract is this binary32 sequence (fmaf fused):     */
-/*   the row is dealt to 32 lanes in 16-element pieces (element k belongs to   */
-/*   lane (k/16) % 32); each lane accumulates ss = fmaf(x, x, ss) over its     */
-/*   elements in increasing k; the 32 partial sums meet in a butterfly         */
-/*   (ss[l] += ss[l ^ off], off = 16, 8, 4, 2, 1);                             */
-/*   rstd = 1 / sqrt(ss / K + eps);   y = bf16_rne( (x * rstd) * w )           */
+/* arithmetic for it; the oracle is the definition in double, rounded once:    */
+/*     y[k] = bf16_rne( x[k] / sqrt( mean_k(x^2) + eps ) * w[k] )              */
 /* ------------------------------------------------------------------------- */
-void orc_rmsnorm_bf16(const uint16_t* x, int64_t rows, int64_t cols, int64_t ld, const uint16_t* w, float eps,
+void orc_rmsnorm_bf16(const uint16_t* x, int64_t rows, int64_t cols, int64_t ld, const uint16_t* w, double eps,
                       uint16_t* y) {
     #pragma omp parallel for schedule(static)
     for (int64_t r = 0; r < rows; ++r) {
-        float ss[32], t[32];
-        for (int l = 0; l < 32; ++l) ss[l] = 0.0f;
+        double ss = 0.0;
         for (int64_t k = 0; k < cols; ++k) {
-            const float v = bf16_to_f32(x[r * ld + k]);
-            const int l = (int)((k / 16) % 32);
-            ss[l] = fmaf(v, v, ss[l]);
+            const double v = (double)bf16_to_f32(x[r * ld + k]);
+            ss += v * v;
         }
-        for (int off = 16; off >= 1; off >>= 1) {
-            for (int l = 0; l < 32; ++l) t[l] = ss[l] + ss[l ^ off];
-            for (int l = 0; l < 32; ++l) ss[l] = t[l];
-        }
-        const float mean = ss[0] / (float)cols;
-        const float rstd = 1.0f / sqrtf(mean + eps);
-        for (int64_t k = 0; k < cols; ++k) {
-            const float v = bf16_to_f32(x[r * ld + k]) * rstd;
-            y[r * cols + k] = orc_f32_to_bf16(v * bf16_to_f32(w[k]));
-        }
+        const double rstd = 1.0 / sqrt(ss / (double)cols + eps);
+        for (int64_t k = 0; k < cols; ++k)
+            y[r * cols + k] = orc_f64_to_bf16((double)bf16_to_f32(x[r * ld + k]) * rstd * (double)bf16_to_f32(w[k]));
     }
 }
 
@@ -280,42 +239,44 @@ void orc_dequantize(const uint8_t* codes, const uint8_t* sf, const float* g_row,
 /* Statistics at NVFP4 granularity (the columns of the paper's Table "stats"): */
 /* max/RMS, kurtosis, share of "1-hot" blocks (block max/RMS > 3, i.e. one     */
 /* value holds more than 9/16 of the block's energy) and the relative error of */
-/* quantizing the tensor alone.  Per block, in binary32 (fmaf fused):          */
-/*   s2 = sum fmaf(x,x,.)   s4 = sum fmaf(x*x, x*x, .)   1-hot: bmax*bmax*16 > 9*s2 */
-/*   se = sum fmaf(e,e,.), e = x - e2m1(code) * (e4m3(s8) * g)                  */
-/* Block results are added up in double.  out: {sum x^2, sum x^4, sum err^2,   */
-/* amax, blocks, 1-hot blocks}.                                                */
+/* quantizing the tensor alone.  Everything is the definition in double:       */
+/*   sum x^2, sum x^4, sum (x - x_hat)^2 with x_hat from orc_quantize /        */
+/*   orc_dequantize's formula, the maximum, and per block: bmax^2 * 16 > 9 * (block's sum x^2). */
+/* (All of x^2, bmax^2 * 16 and 9 * sum are exact in double for bf16 inputs,   */
+/* so the 1-hot count has no rounding in it.)                                  */
+/* out: {sum x^2, sum x^4, sum err^2, amax, blocks, 1-hot blocks}.             */
 /* ------------------------------------------------------------------------- */
 int orc_stats(const uint16_t* x, int64_t rows, int64_t cols, int64_t ld, float g, double* out) {
     if (cols % 16 != 0) return 1;
-    double t2 = 0.0, t4 = 0.0, te = 0.0, hot = 0.0;
-    float amax = 0.0f;
-    const float c1 = 1.0f / (6.0f * g);
+    double t2 = 0.0, t4 = 0.0, te = 0.0, hot = 0.0, amax = 0.0;
+    const float c1 = 1.0f / (6.0f * g);                         /* as in orc_quantize */
     for (int64_t r = 0; r < rows; ++r)
         for (int64_t b = 0; b < cols / 16; ++b) {
             const uint16_t* xb = x + r * ld + b * 16;
-            float s2 = 0.0f, s4 = 0.0f, se = 0.0f, bmax = 0.0f;
+            double s2 = 0.0, bmax = 0.0;
+            float bmaxf = 0.0f;
             for (int i = 0; i < 16; ++i) {
-                const float v = bf16_to_f32(xb[i]);
-                const float q = v * v;
-                s2 = fmaf(v, v, s2);
-                s4 = fmaf(q, q, s4);
-                if (fabsf(v) > bmax) bmax = fabsf(v);
+                const double v = (double)bf16_to_f32(xb[i]);
+                s2 += v * v;
+                t4 += (v * v) * (v * v);
+                if (fabs(v) > bmax) { bmax = fabs(v); bmaxf = fabsf(bf16_to_f32(xb[i])); }
             }
+            t2 += s2;
             if (bmax > amax) amax = bmax;
-            if ((bmax * bmax) * 16.0f > 9.0f * s2) hot += 1.0;
-            const uint8_t s8 = orc_e4m3_encode(bmax * c1);
-            const float d = orc_e4m3_decode(s8) * g;
-            const float qinv = 1.0f / d;
+            if (bmax * bmax * 16.0 > 9.0 * s2) hot += 1.0;
+            /* quantize this block exactly as orc_quantize does, dequantize as orc_dequantize does */
+            const uint8_t s8 = orc_e4m3_encode(bmaxf * c1);
+            const float sdec = orc_e4m3_decode(s8);
+            const float q = 1.0f / (sdec * g);
             for (int i = 0; i < 16; ++i) {
-                const float v = bf16_to_f32(xb[i]);
-                const float xh = (s8 == 0) ? 0.0f : orc_e2m1_decode(orc_e2m1_encode(v * qinv)) * d;
-                const float e = v - xh;
-                se = fmaf(e, e, se);
+                const float xv = bf16_to_f32(xb[i]);
+                const double xh = (s8 == 0) ? 0.0
+                    : (double)orc_e2m1_decode(orc_e2m1_encode(xv * q)) * (double)sdec * (double)g;
+                const double e = (double)xv - xh;
+                te += e * e;
             }
-            t2 += (double)s2; t4 += (double)s4; te += (double)se;
         }
-    out[0] = t2; out[1] = t4; out[2] = te; out[3] = (double)amax;
+    out[0] = t2; out[1] = t4; out[2] = te; out[3] = amax;
     out[4] = (double)(rows * (cols / 16)); out[5] = hot;
     return 0;
 }

@@ -62,9 +62,9 @@ def lib() -> ctypes.CDLL:
     L.nvfp4_quantize_act.restype = i32
     L.nvfp4_quantize_act.argtypes = [vp, i64, i64, i64, vp, vp, vp, i32, vp]
     L.nvfp4_swiglu_quantize.restype = i32
-    L.nvfp4_swiglu_quantize.argtypes = [vp, i64, i64, i64, vp, vp, vp, i32, vp]
+    L.nvfp4_swiglu_quantize.argtypes = [vp, i64, i64, i64, vp, vp, vp, i32, vp, vp]
     L.nvfp4_rmsnorm_quantize.restype = i32
-    L.nvfp4_rmsnorm_quantize.argtypes = [vp, i64, i64, i64, vp, ctypes.c_float, vp, vp, vp, i32, vp]
+    L.nvfp4_rmsnorm_quantize.argtypes = [vp, i64, i64, i64, vp, ctypes.c_float, vp, vp, vp, i32, vp, vp]
     L.nvfp4_quantize_weight.restype = i32
     L.nvfp4_quantize_weight.argtypes = [vp, i64, i64, i64, segp, i32, vp, i32, vp, vp, i32, vp]
     L.nvfp4_harmonize_scales.restype = i32
@@ -183,26 +183,32 @@ def nvfp4_quantize_act(x: torch.Tensor, g: torch.Tensor, layout: int = SF_MMA, o
     return codes, sf
 
 
-def nvfp4_swiglu_quantize(gate_up: torch.Tensor, g: torch.Tensor, layout: int = SF_MMA, out=None, stream=None):
-    """bf16 [M, 2I] (gate | up) -> NVFP4 of bf16(silu(gate) * up): (codes u8 [M, I/2], scale bytes)."""
+def nvfp4_swiglu_quantize(gate_up: torch.Tensor, g: torch.Tensor, layout: int = SF_MMA, out=None, stream=None,
+                          h_out: Optional[torch.Tensor] = None):
+    """bf16 [M, 2I] (gate | up) -> NVFP4 of bf16(silu(gate) * up): (codes u8 [M, I/2], scale bytes).
+    ``h_out`` (bf16 [M, I], contiguous; testing aid) also receives the tensor that was quantized."""
     assert gate_up.is_cuda and gate_up.dtype == torch.bfloat16 and gate_up.dim() == 2 and gate_up.stride(1) == 1
     M, two_i = gate_up.shape
     inner = two_i // 2
+    assert h_out is None or (h_out.dtype == torch.bfloat16 and h_out.shape == (M, inner) and h_out.is_contiguous())
     codes, sf = out if out is not None else alloc_quantized(M, inner, gate_up.device, layout)
     _check(lib().nvfp4_swiglu_quantize(_ptr(gate_up), M, inner, gate_up.stride(0), _ptr(g), _ptr(codes), _ptr(sf),
-                                       layout, _stream(stream)), "nvfp4_swiglu_quantize")
+                                       layout, _ptr(h_out), _stream(stream)), "nvfp4_swiglu_quantize")
     return codes, sf
 
 
 def nvfp4_rmsnorm_quantize(x: torch.Tensor, weight: torch.Tensor, eps: float, g: torch.Tensor, layout: int = SF_MMA,
-                           out=None, stream=None):
-    """bf16 [M, K], gain bf16 [K] -> NVFP4 of bf16(RMSNorm(x) * weight): (codes, scale bytes)."""
+                           out=None, stream=None, y_out: Optional[torch.Tensor] = None):
+    """bf16 [M, K], gain bf16 [K] -> NVFP4 of bf16(RMSNorm(x) * weight): (codes, scale bytes).
+    ``y_out`` (bf16 [M, K], contiguous; testing aid) also receives the tensor that was quantized."""
     assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
     assert weight.dtype == torch.bfloat16 and weight.numel() == x.shape[1] and weight.is_contiguous()
     M, K = x.shape
+    assert y_out is None or (y_out.dtype == torch.bfloat16 and y_out.shape == (M, K) and y_out.is_contiguous())
     codes, sf = out if out is not None else alloc_quantized(M, K, x.device, layout)
     _check(lib().nvfp4_rmsnorm_quantize(_ptr(x), M, K, x.stride(0), _ptr(weight), ctypes.c_float(eps), _ptr(g),
-                                        _ptr(codes), _ptr(sf), layout, _stream(stream)), "nvfp4_rmsnorm_quantize")
+                                        _ptr(codes), _ptr(sf), layout, _ptr(y_out), _stream(stream)),
+           "nvfp4_rmsnorm_quantize")
     return codes, sf
 
 
@@ -282,7 +288,8 @@ def nvfp4_linear_bf16(x, g_a, w_codes, w_sf, segments, g_seg, workspace, out=Non
     return out
 
 
-STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
+STATIC_SCRATCH_BYTES = 12 * 1024 * 1024
+SPLIT_RESERVE_BYTES = 5 * 1024 * 1024      # split-K part of every workspace, directly behind the 256-byte status block
 
 
 def nvfp4_linear_bf16_static(x, g_a, w_codes, w_sf, segments, g_seg, out=None, out_f32: bool = False,
@@ -308,7 +315,8 @@ def nvfp4_linear_bf16_static(x, g_a, w_codes, w_sf, segments, g_seg, out=None, o
 
 
 def static_status(stream=None) -> int:
-    """Status word of the library's static scratch (synchronises the stream)."""
+    """Status word of the library's static scratch (synchronises the stream); a failure also
+    clears the word and re-zeroes the split-K part of the array."""
     return int(lib().nvfp4_static_status(_stream(stream)))
 
 
@@ -317,5 +325,6 @@ def workspace_reset(workspace: torch.Tensor, stream=None) -> None:
 
 
 def device_status(workspace: torch.Tensor, stream=None) -> int:
-    """Synchronises the stream; 0 = ok, 8 = a bounded in-kernel wait ran out."""
+    """Synchronises the stream; 0 = ok, 8 = a bounded in-kernel wait ran out, 10 = a global scale
+    read on the device was not finite and positive."""
     return int(lib().nvfp4_device_status(_ptr(workspace), _stream(stream)))

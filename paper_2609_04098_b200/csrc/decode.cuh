@@ -30,6 +30,7 @@ struct DecodeParams {
     const float* g_seg;
     void* y;
     int64_t ldy;
+    uint32_t* status;        // first word of the workspace (a bad global scale is reported there)
     int32_t M, N, K;
     uint32_t flags;
     int32_t nseg;
@@ -108,6 +109,16 @@ decode_gemv_kernel(const __grid_constant__ DecodeParams p) {
         }
     };
     if (items > 0) load_item(0, 0);
+    if (blockIdx.x == 0 && warp == 0) {
+        // global scales must be finite and positive; anything else is reported, not repaired
+        const float ga = __ldg(p.g_a);
+        bool bad = !(ga > 0.0f && ga <= 3.402823466e38f);
+        for (int i = lane; i < p.nseg; i += 32) {
+            const float gs = __ldg(p.g_seg + i);
+            bad = bad || !(gs > 0.0f && gs <= 3.402823466e38f);
+        }
+        if (__any_sync(0xffffffffu, bad) && lane == 0) atomicExch(p.status, static_cast<uint32_t>(NVFP4_ERR_SCALE));
+    }
 
     // ---- 1. quantize the activation rows (every CTA its own copy)
     {

@@ -64,23 +64,7 @@ struct GemmParams {
     int32_t nseg;
     int32_t seg_end[NVFP4_MAX_SEGMENTS];
     uint64_t wait_limit_ns;
-#ifdef NVFP4_PROBE
-    uint32_t probe;              // timing experiments only (results are wrong): see the bits below
-    unsigned long long* trace;   // [role][256] globaltimer stamps written by block 0
-#endif
 };
-#ifdef NVFP4_PROBE
-#define NVFP4_PROBE_BIT(p, b) (((p).probe >> (b)) & 1u)
-#define NVFP4_TRACE(p, role, idx)                                                        \
-    do {                                                                                 \
-        if ((p).trace != nullptr && blockIdx.x == 0 && (idx) < 256u)                     \
-            (p).trace[(role) * 256 + (idx)] = ptx::globaltimer_ns();                     \
-    } while (0)
-#else
-#define NVFP4_PROBE_BIT(p, b) 0u
-#define NVFP4_TRACE(p, role, idx) do {} while (0)
-#endif
-// probe bits: 0 no MMA, 1 no code loads, 2 no scale loads, 3 no scale copies to TMEM, 4 no epilogue stores
 
 constexpr int kGemmThreads = 224;
 constexpr int kBM = 128;
@@ -217,11 +201,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             ptx::prefetch_tensormap(tm_sf);
             const uint32_t code_off = is_a ? 0u : C::A_BYTES;
             const uint32_t sf_off = C::A_BYTES + C::B_BYTES + (is_a ? 0u : C::SFA_BYTES);
-            uint32_t tx = is_a ? (C::A_BYTES + C::SFA_BYTES) : (C::B_BYTES + C::SFB_BYTES);
-#ifdef NVFP4_PROBE
-            if (NVFP4_PROBE_BIT(p, 1)) tx -= is_a ? C::A_BYTES : C::B_BYTES;
-            if (NVFP4_PROBE_BIT(p, 2)) tx -= is_a ? C::SFA_BYTES : C::SFB_BYTES;
-#endif
+            const uint32_t tx = is_a ? (C::A_BYTES + C::SFA_BYTES) : (C::B_BYTES + C::SFB_BYTES);
             uint32_t it = 0;
             bool ok = true;
             for (uint32_t t = 0; ok && t < my_tiles; ++t) {
@@ -234,18 +214,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 for (int32_t kt = ks * p.k_per_split; kt < kt_end; ++kt, ++it) {
                     const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
                     if (!ptx::mbar_wait_bounded(&empty[s], ph ^ 1u, abort_flag, p.wait_limit_ns, peer_abort)) { ok = false; break; }
-                    if (is_a) NVFP4_TRACE(p, 0, it);
                     uint8_t* st = smem + s * C::STAGE_BYTES;
                     // rows / bands / k-atoms past the tensor are zero-filled by TMA
                     if (PAIR) {
                         const uint32_t bar = leader_full + s * 8u;
                         ptx::mbar_arrive_expect_tx_cluster(bar, tx);
-                        if (!NVFP4_PROBE_BIT(p, 1)) ptx::tma_load_2d_pair(st + code_off, tm_codes, kt * kBKBytes, code_row, bar);
-                        if (!NVFP4_PROBE_BIT(p, 2)) ptx::tma_load_3d_pair(st + sf_off, tm_sf, 0, kt * kStepsPerStage, sf_band, bar);
+                        ptx::tma_load_2d_pair(st + code_off, tm_codes, kt * kBKBytes, code_row, bar);
+                        ptx::tma_load_3d_pair(st + sf_off, tm_sf, 0, kt * kStepsPerStage, sf_band, bar);
                     } else {
                         ptx::mbar_arrive_expect_tx(&full[s], tx);
-                        if (!NVFP4_PROBE_BIT(p, 1)) ptx::tma_load_2d(st + code_off, tm_codes, kt * kBKBytes, code_row, &full[s]);
-                        if (!NVFP4_PROBE_BIT(p, 2)) ptx::tma_load_3d(st + sf_off, tm_sf, 0, kt * kStepsPerStage, sf_band, &full[s]);
+                        ptx::tma_load_2d(st + code_off, tm_codes, kt * kBKBytes, code_row, &full[s]);
+                        ptx::tma_load_3d(st + sf_off, tm_sf, 0, kt * kStepsPerStage, sf_band, &full[s]);
                     }
                 }
             }
@@ -301,7 +280,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                         ptx::tc_fence_after();
                     }
                     have_full = false;
-                    if (leader) NVFP4_TRACE(p, 2, it);
                     const uint32_t st_enc = smem_enc + s * (C::STAGE_BYTES >> 4);
                     const uint32_t sfa_t = tmem_base + C::SFA_COL0 + (C::SF_SETS == 1 ? 0 : s) * C::SFA_SET_COLS;
                     const uint32_t sfb_t = tmem_base + C::SFB_COL0 + (C::SF_SETS == 1 ? 0 : s) * C::SFB_SET_COLS;
@@ -318,7 +296,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                             }
                             // this step's scale atoms: shared -> TMEM (32 rows x 16 bytes each, replicated into
                             // the four lane quarters), then the MMA that reads them
-                            if (!NVFP4_PROBE_BIT(p, 3) && leader) {
+                            if (leader) {
                                 const uint32_t sf_enc = st_enc + ((C::A_BYTES + C::B_BYTES + j * 512) >> 4);
                                 if (PAIR) {
                                     ptx::tc_cp_32x128b_warpx4_pair(sfa_t + j * 4, desc(sf_enc, kScaleHi));
@@ -334,7 +312,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                                                                   desc(sf_enc + ((C::SFA_BYTES + kStepsPerStage * 512) >> 4), kScaleHi));
                                 }
                             }
-                            if (!NVFP4_PROBE_BIT(p, 0) && leader) {
+                            if (leader) {
                                 // advancing K by 64 elements = 32 bytes inside the 128-byte swizzle row
                                 const uint64_t a_desc = desc((st_enc + j * 2) | kCodeLoFlags, kCodeHi);
                                 const uint64_t b_desc = desc((st_enc + (C::A_BYTES >> 4) + j * 2) | kCodeLoFlags, kCodeHi);
@@ -353,7 +331,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                             ptx::tc_commit(&empty[s]);
                             if (last_kt) ptx::tc_commit(&tfull[acc]);
                         }
-                        NVFP4_TRACE(p, 3, it);
                     }
                     ++it;
                     if (last_kt) { kt = 0; ++tl; } else { ++kt; }
@@ -375,13 +352,21 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         const bool use_tma = p.tma_store != 0u;
         const uint32_t leader_tempty = PAIR ? ptx::mapa_shared(ptx::smem_u32(tempty), 0u) : ptx::smem_u32(tempty);
         if (use_tma && lane == 0) ptx::prefetch_tensormap(&tmY);
+        if (blockIdx.x == 0 && warp == 0) {
+            // global scales must be finite and positive; anything else is reported, not repaired
+            bool bad = !(g_a > 0.0f && g_a <= 3.402823466e38f);
+            for (int i = lane; i < p.nseg; i += 32) {
+                const float gs = __ldg(p.g_seg + i);
+                bad = bad || !(gs > 0.0f && gs <= 3.402823466e38f);
+            }
+            if (__any_sync(0xffffffffu, bad) && lane == 0) atomicExch(p.status, static_cast<uint32_t>(NVFP4_ERR_SCALE));
+        }
         uint32_t pieces_stored = 0;
         for (uint32_t t = 0; t < my_tiles; ++t) {
             int32_t um, un, ks;
             tile_of(t, um, un, ks);
             const int32_t n0 = un * BN;
             const uint32_t acc = t & 1u, aph = (t >> 1) & 1u;
-            if (warp == 0 && lane == 0) NVFP4_TRACE(p, 7, t);
             // global scale of columns n0 + 32 i + lane, i = 0 .. BN/32-1, in registers
             float areg[BN / 32];
 #pragma unroll
@@ -402,7 +387,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             ok = __shfl_sync(0xffffffffu, static_cast<int>(ok), 0) != 0;
             if (!ok) break;
             ptx::tc_fence_after();
-            if (warp == 0 && lane == 0) NVFP4_TRACE(p, 6, t);
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * C::ACC_STRIDE;
             const int32_t row0 = (PAIR ? 2 * um + static_cast<int32_t>(rank) : um) * kBM + quarter * 32;
             constexpr int NP = BN / kOutPieceCols;
@@ -518,7 +502,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     }
                 }
                 const int32_t col0 = n0 + pc * kOutPieceCols;
-                if (col0 >= p.N || row0 >= p.M || NVFP4_PROBE_BIT(p, 4)) continue;        // warp-uniform
+                if (col0 >= p.N || row0 >= p.M) continue;        // warp-uniform
                 float v[64];
 #pragma unroll
                 for (int j = 0; j < 64; ++j)

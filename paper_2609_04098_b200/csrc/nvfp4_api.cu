@@ -204,10 +204,7 @@ nvfp4_status launch_gemm(const GemmMaps& tm, GemmParams& p, int sm_count, cudaSt
     {
         // rows of A kept live per raster group: about 32 MB of codes and scales (a quarter of L2)
         const int64_t unit_bytes = static_cast<int64_t>(PAIR ? 256 : 128) * (p.K / 2 + p.K / 16);
-        int64_t budget = 32ll << 20;
-#ifdef NVFP4_PROBE
-        if (getenv("NVFP4_GROUP_MB")) budget = static_cast<int64_t>(atoi(getenv("NVFP4_GROUP_MB"))) << 20;
-#endif
+        const int64_t budget = 32ll << 20;
         int64_t g = budget / (unit_bytes > 0 ? unit_bytes : 1);
         if (g < 1) g = 1;
         if (g > m_units) g = m_units;
@@ -270,7 +267,7 @@ template <bool MMA, int MODE>
 nvfp4_status launch_quantize(const uint16_t* x, int64_t M, int64_t K, int64_t ld, const float* d_g,
                              const SegTable& segs, uint8_t* d_codes, uint8_t* d_sf, int64_t chunks, int64_t per_unit,
                              int64_t units_per_row, int64_t units, int sm_count, cudaStream_t stream,
-                             const uint16_t* aux, float eps) {
+                             const uint16_t* aux, float eps, uint16_t* h_out) {
     constexpr int kUnroll = 2;
     // persistent grid: exactly what is resident at once, so that no partial second wave forms
     static std::atomic<int> per_sm_cache{0};
@@ -288,9 +285,36 @@ nvfp4_status launch_quantize(const uint16_t* x, int64_t M, int64_t K, int64_t ld
     if (blocks > max_blocks) blocks = max_blocks;
     if (blocks < 1) blocks = 1;
     quantize_kernel<MMA, kUnroll, MODE><<<static_cast<int>(blocks), 256, 0, stream>>>(
-        x, static_cast<int32_t>(M), static_cast<int32_t>(K), ld, d_g, segs, aux, eps, d_codes, d_sf,
+        x, static_cast<int32_t>(M), static_cast<int32_t>(K), ld, d_g, segs, aux, eps, d_codes, d_sf, h_out,
         static_cast<int32_t>(chunks), static_cast<int32_t>(per_unit), static_cast<int32_t>(units_per_row),
         static_cast<int32_t>(units));
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+}
+
+// RMSNorm -> quantize with the row held in registers by W warps (rows of up to 8 * kRmsChunks chunks)
+template <bool MMA, int W>
+nvfp4_status launch_rmsnorm(const uint16_t* x, int64_t M, int64_t rows_total, int64_t K, int64_t ld, const float* d_g,
+                            const uint16_t* gain, float eps, uint8_t* d_codes, uint8_t* d_sf, uint16_t* y_out,
+                            int64_t chunks, int sm_count, cudaStream_t stream) {
+    static std::atomic<int> per_sm_cache{0};
+    int per_sm = per_sm_cache.load(std::memory_order_relaxed);
+    if (per_sm == 0) {
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rmsnorm_quantize_kernel<MMA, W>, 256, 0) != cudaSuccess ||
+            per_sm < 1) {
+            cudaGetLastError();
+            per_sm = 2;
+        }
+        per_sm_cache.store(per_sm, std::memory_order_relaxed);
+    }
+    constexpr int kGroups = 8 / W;
+    int64_t blocks = (rows_total + kGroups - 1) / kGroups;
+    const int64_t max_blocks = static_cast<int64_t>(sm_count) * per_sm;
+    if (blocks > max_blocks) blocks = max_blocks;
+    if (blocks < 1) blocks = 1;
+    rmsnorm_quantize_kernel<MMA, W><<<static_cast<int>(blocks), 256, 0, stream>>>(
+        x, static_cast<int32_t>(M), static_cast<int32_t>(rows_total), static_cast<int32_t>(K), ld, d_g, gain, eps,
+        d_codes, d_sf, y_out, static_cast<int32_t>(chunks), static_cast<int32_t>((chunks + W - 1) / W));
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
@@ -298,9 +322,26 @@ nvfp4_status launch_quantize(const uint16_t* x, int64_t M, int64_t K, int64_t ld
 nvfp4_status quantize_impl(const void* d_x, int64_t M, int64_t K, int64_t ld, const float* d_g,
                            const SegTable& segs, uint8_t* d_codes, uint8_t* d_sf, nvfp4_sf_layout layout,
                            const DeviceInfo& info, cudaStream_t stream, int mode = kQuantPlain,
-                           const uint16_t* aux = nullptr, float eps = 0.0f) {
+                           const uint16_t* aux = nullptr, float eps = 0.0f, uint16_t* h_out = nullptr) {
     const int64_t chunks = (K + 511) / 512;              // 512 elements = one block per lane
     if (M >= (1ll << 31) || K >= (1ll << 31)) return NVFP4_ERR_SHAPE;
+    if (mode == kQuantRmsnorm && chunks <= 8 * kRmsChunks) {
+        const uint16_t* xr = reinterpret_cast<const uint16_t*>(d_x);
+        const int64_t rows_all = (layout == NVFP4_SF_MMA) ? (M + 127) / 128 * 128 : M;
+        const bool mma_l = layout == NVFP4_SF_MMA;
+        int w = 1;
+        while (w < 8 && (chunks + w - 1) / w > kRmsChunks) w *= 2;
+        if (w == 1 && chunks >= 2 && chunks % 2 == 0) w = 2;       // shorter dependency chain per row, same registers
+#define NVFP4_LAUNCH_R(MMA_, W_) \
+    launch_rmsnorm<MMA_, W_>(xr, M, rows_all, K, ld, d_g, aux, eps, d_codes, d_sf, h_out, chunks, info.sm_count, stream)
+        switch (w) {
+            case 1: return mma_l ? NVFP4_LAUNCH_R(true, 1) : NVFP4_LAUNCH_R(false, 1);
+            case 2: return mma_l ? NVFP4_LAUNCH_R(true, 2) : NVFP4_LAUNCH_R(false, 2);
+            case 4: return mma_l ? NVFP4_LAUNCH_R(true, 4) : NVFP4_LAUNCH_R(false, 4);
+            default: return mma_l ? NVFP4_LAUNCH_R(true, 8) : NVFP4_LAUNCH_R(false, 8);
+        }
+#undef NVFP4_LAUNCH_R
+    }
     // a unit = up to `per_unit` consecutive chunks of one row, handled by one warp
     constexpr int kUnroll = 2;      // matches launch_quantize
     const int64_t resident_warps = static_cast<int64_t>(info.sm_count) * 40;   // 5 blocks of 8 warps per SM
@@ -315,7 +356,7 @@ nvfp4_status quantize_impl(const void* d_x, int64_t M, int64_t K, int64_t ld, co
     const bool mma = layout == NVFP4_SF_MMA;
 #define NVFP4_LAUNCH_Q(MMA_, MODE_)                                                                          \
     launch_quantize<MMA_, MODE_>(x, M, K, ld, d_g, segs, d_codes, d_sf, chunks, per_unit, units_per_row, units, \
-                                 info.sm_count, stream, aux, eps)
+                                 info.sm_count, stream, aux, eps, h_out)
     if (mode == kQuantSwiglu) return mma ? NVFP4_LAUNCH_Q(true, kQuantSwiglu) : NVFP4_LAUNCH_Q(false, kQuantSwiglu);
     if (mode == kQuantRmsnorm) return mma ? NVFP4_LAUNCH_Q(true, kQuantRmsnorm) : NVFP4_LAUNCH_Q(false, kQuantRmsnorm);
     return mma ? NVFP4_LAUNCH_Q(true, kQuantPlain) : NVFP4_LAUNCH_Q(false, kQuantPlain);
@@ -333,8 +374,12 @@ nvfp4_status check_quantize_args(const void* d_x, int64_t rows, int64_t K, int64
 }
 
 constexpr size_t kStatusBytes = 256;
+constexpr size_t kSplitReserve = NVFP4_SPLIT_RESERVE_BYTES;
 
-// split-K area of a workspace (after the status block): counters, then fp32 partial sums
+// Split-K area of a workspace: counters, then fp32 partial sums.  It always starts directly behind
+// the status block, whatever the problem size, and never reaches past the reserve, so that nothing
+// else the library keeps in a workspace (the quantized activations of nvfp4_linear_bf16 live behind
+// the reserve) can ever land on it: it stays zero between calls by construction.
 struct SplitArea {
     size_t counters_bytes = 0, partial_bytes = 0;
     int64_t ldp = 0;
@@ -347,7 +392,7 @@ SplitArea split_area(int64_t M, int64_t N) {
     a.counters_bytes = (static_cast<size_t>(m_tiles * n_tiles * 4) * sizeof(uint32_t) + 255) & ~static_cast<size_t>(255);
     a.ldp = n_tiles * 128;
     a.partial_bytes = static_cast<size_t>(m_tiles * 128) * static_cast<size_t>(a.ldp) * sizeof(float);
-    if (a.partial_bytes > (64u << 20)) return SplitArea();
+    if (a.total() > kSplitReserve) return SplitArea();         // too large for the reserve: no split-K
     return a;
 }
 
@@ -437,17 +482,19 @@ nvfp4_status nvfp4_quantize_weight(const void* d_w, int64_t N, int64_t K, int64_
 }
 
 nvfp4_status nvfp4_swiglu_quantize(const void* d_gate_up, int64_t M, int64_t inner, int64_t ld, const float* d_g,
-                                   uint8_t* d_codes, uint8_t* d_sf, nvfp4_sf_layout layout, void* stream) {
+                                   uint8_t* d_codes, uint8_t* d_sf, nvfp4_sf_layout layout, void* d_h, void* stream) {
     nvfp4_status st = check_quantize_args(d_gate_up, M, inner, ld, d_g, d_codes, d_sf, layout);
     if (st != NVFP4_OK) return st;
     if (ld < 2 * inner) return NVFP4_ERR_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(d_h) & 31u) != 0) return NVFP4_ERR_ALIGN;
     if (M == 0) return NVFP4_OK;
     DeviceInfo info;
     st = check_arch(info);
     if (st != NVFP4_OK) return st;
     SegTable segs;
     std::memset(&segs, 0, sizeof(segs));
-    return quantize_impl(d_gate_up, M, inner, ld, d_g, segs, d_codes, d_sf, layout, info, as_stream(stream), kQuantSwiglu);
+    return quantize_impl(d_gate_up, M, inner, ld, d_g, segs, d_codes, d_sf, layout, info, as_stream(stream), kQuantSwiglu,
+                         nullptr, 0.0f, reinterpret_cast<uint16_t*>(d_h));
 }
 
 nvfp4_status nvfp4_harmonize_scales(const uint8_t* d_sf_in, int64_t N, int64_t K, nvfp4_sf_layout layout,
@@ -485,11 +532,11 @@ nvfp4_status nvfp4_harmonize_scales(const uint8_t* d_sf_in, int64_t N, int64_t K
 
 nvfp4_status nvfp4_rmsnorm_quantize(const void* d_x, int64_t M, int64_t K, int64_t ld, const void* d_weight, float eps,
                                     const float* d_g, uint8_t* d_codes, uint8_t* d_sf, nvfp4_sf_layout layout,
-                                    void* stream) {
+                                    void* d_y, void* stream) {
     nvfp4_status st = check_quantize_args(d_x, M, K, ld, d_g, d_codes, d_sf, layout);
     if (st != NVFP4_OK) return st;
     if (d_weight == nullptr) return NVFP4_ERR_NULL;
-    if ((reinterpret_cast<uintptr_t>(d_weight) & 31u) != 0) return NVFP4_ERR_ALIGN;
+    if (((reinterpret_cast<uintptr_t>(d_weight) | reinterpret_cast<uintptr_t>(d_y)) & 31u) != 0) return NVFP4_ERR_ALIGN;
     if (!(eps >= 0.0f)) return NVFP4_ERR_SHAPE;
     if (M == 0) return NVFP4_OK;
     DeviceInfo info;
@@ -498,7 +545,7 @@ nvfp4_status nvfp4_rmsnorm_quantize(const void* d_x, int64_t M, int64_t K, int64
     SegTable segs;
     std::memset(&segs, 0, sizeof(segs));
     return quantize_impl(d_x, M, K, ld, d_g, segs, d_codes, d_sf, layout, info, as_stream(stream), kQuantRmsnorm,
-                         reinterpret_cast<const uint16_t*>(d_weight), eps);
+                         reinterpret_cast<const uint16_t*>(d_weight), eps, reinterpret_cast<uint16_t*>(d_y));
 }
 
 nvfp4_status nvfp4_tensor_stats(const void* d_x, int64_t rows, int64_t cols, int64_t ld, const float* d_g,
@@ -625,10 +672,6 @@ nvfp4_status linear_impl(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const 
         const uint64_t lim = g_wait_limit_ns.load(std::memory_order_relaxed);
         p.wait_limit_ns = lim != 0 ? lim : kWaitLimitNs;
     }
-#ifdef NVFP4_PROBE
-    p.probe = getenv("NVFP4_PROBE") ? static_cast<uint32_t>(atoi(getenv("NVFP4_PROBE"))) : 0u;
-    p.trace = getenv("NVFP4_TRACE_PTR") ? reinterpret_cast<unsigned long long*>(strtoull(getenv("NVFP4_TRACE_PTR"), nullptr, 16)) : nullptr;
-#endif
     cudaStream_t s = as_stream(stream);
     switch (bn) {
         case 128: return launch_gemm<128, 5, false>(tm, p, info.sm_count, s);
@@ -663,14 +706,75 @@ nvfp4_status launch_decode(const DecodeParams& p, int sm_count, cudaStream_t str
     return cudaGetLastError() == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
 
-// workspace of the fused call: [status][codes][scales][optional split-K area]
+// workspace of the fused call: [status][split-K reserve][codes][scales]; every part at an offset
+// that does not depend on the problem size
 size_t fused_codes_bytes(int64_t M, int64_t K) {        // rows padded to whole 128-row tiles
     const int64_t m_pad = (M + 127) / 128 * 128;
     return (static_cast<size_t>(m_pad) * static_cast<size_t>(K / 2) + 255) & ~static_cast<size_t>(255);
 }
+constexpr size_t kFusedCodesOffset = kStatusBytes + kSplitReserve;
 size_t fused_min_bytes(int64_t M, int64_t K) {
     const size_t sf = (nvfp4_sf_bytes(M, K, NVFP4_SF_MMA) + 255) & ~static_cast<size_t>(255);
-    return kStatusBytes + fused_codes_bytes(M, K) + sf;
+    return kFusedCodesOffset + fused_codes_bytes(M, K) + sf;
+}
+
+// nvfp4_linear_bf16 on a workspace of the layout above; every argument is checked before
+// anything is enqueued
+nvfp4_status linear_bf16_impl(const void* d_x, int64_t ldx, const float* d_g_a, int64_t M, int64_t K,
+                              const uint8_t* d_w_codes, const uint8_t* d_w_sf, int64_t N,
+                              const nvfp4_segment* segs, const float* d_g_seg, int nseg, void* d_y, int64_t ldy,
+                              uint32_t flags, void* d_workspace, size_t workspace_bytes, void* stream) {
+    if (d_workspace == nullptr) return NVFP4_ERR_WORKSPACE;
+    if (M < 0 || N < 0 || K <= 0 || (K % 64) != 0) return NVFP4_ERR_SHAPE;
+    if (d_x == nullptr || d_g_a == nullptr || d_w_codes == nullptr || d_w_sf == nullptr || d_g_seg == nullptr ||
+        d_y == nullptr)
+        return NVFP4_ERR_NULL;
+    if (ldx < K || ldy < N || M >= (1ll << 31) - 256 || N >= (1ll << 31) - 256 || K >= (1ll << 31)) return NVFP4_ERR_SHAPE;
+    if ((flags & ~(NVFP4_OUT_F32 | NVFP4_WS_ZEROED)) != 0u) return NVFP4_ERR_SHAPE;
+    nvfp4_status st = check_segments(segs, nseg, N);
+    if (N == 0 && segs != nullptr) st = NVFP4_OK;
+    if (st != NVFP4_OK) return st;
+    if ((reinterpret_cast<uintptr_t>(d_x) & 31u) != 0 || (ldx % 16) != 0 || !aligned16(d_w_codes) || !aligned16(d_w_sf) ||
+        !aligned16(d_workspace))
+        return NVFP4_ERR_ALIGN;
+    const size_t min_bytes = fused_min_bytes(M, K);
+    if (workspace_bytes < min_bytes) return NVFP4_ERR_WORKSPACE;
+    if (M == 0 || N == 0) return NVFP4_OK;
+    // measured on B200 (5120 -> 6144, CUDA-graph replay): 1 / 2 tokens are faster through the
+    // weight-streaming kernel; from 3 tokens on the tensor cores win
+    if (M <= 2 && g_variant.load(std::memory_order_relaxed) == 0 && decode_smem_bytes(M, K) <= 200 * 1024) {
+        // decode-sized batch: one weight-streaming kernel; of the workspace only the status word is used
+        DeviceInfo info;
+        st = check_arch(info);
+        if (st != NVFP4_OK) return st;
+        DecodeParams dp;
+        std::memset(&dp, 0, sizeof(dp));
+        dp.x = reinterpret_cast<const uint16_t*>(d_x);
+        dp.ldx = ldx;
+        dp.g_a = d_g_a;
+        dp.w_codes = d_w_codes;
+        dp.w_sf = d_w_sf;
+        dp.g_seg = d_g_seg;
+        dp.y = d_y;
+        dp.ldy = ldy;
+        dp.status = reinterpret_cast<uint32_t*>(d_workspace);
+        dp.M = static_cast<int32_t>(M);
+        dp.N = static_cast<int32_t>(N);
+        dp.K = static_cast<int32_t>(K);
+        dp.flags = flags;
+        dp.nseg = nseg;
+        for (int i = 0; i < nseg; ++i) dp.seg_end[i] = static_cast<int32_t>(segs[i].col_begin + segs[i].col_count);
+        cudaStream_t s = as_stream(stream);
+        if (M == 1) return launch_decode<1>(dp, info.sm_count, s);
+        return launch_decode<2>(dp, info.sm_count, s);
+    }
+    uint8_t* ws = reinterpret_cast<uint8_t*>(d_workspace);
+    uint8_t* codes = ws + kFusedCodesOffset;
+    uint8_t* sf = codes + fused_codes_bytes(M, K);
+    st = nvfp4_quantize_act(d_x, M, K, ldx, d_g_a, codes, sf, NVFP4_SF_MMA, stream);
+    if (st != NVFP4_OK) return st;
+    return linear_impl(codes, sf, d_g_a, M, K, d_w_codes, d_w_sf, N, segs, d_g_seg, nseg, d_y, ldy, flags, d_workspace,
+                       kStatusBytes, ws + kStatusBytes, kSplitReserve, stream, (M + 127) / 128 * 128);
 }
 }  // namespace
 
@@ -685,70 +789,24 @@ nvfp4_status nvfp4_linear(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const
     if (d_workspace != nullptr && workspace_bytes > kStatusBytes) {
         split = reinterpret_cast<uint8_t*>(d_workspace) + kStatusBytes;
         split_bytes = workspace_bytes - kStatusBytes;
+        if (split_bytes > kSplitReserve) split_bytes = kSplitReserve;
     }
     return linear_impl(d_a_codes, d_a_sf, d_g_a, M, K, d_w_codes, d_w_sf, N, segs, d_g_seg, nseg, d_y, ldy, flags,
                        d_workspace, workspace_bytes, split, split_bytes, stream);
 }
 
 size_t nvfp4_linear_bf16_workspace_bytes(int64_t M, int64_t N, int64_t K, int nseg) {
-    (void)nseg;
+    (void)N; (void)nseg;
     if (M < 0 || K < 0 || (K % 16) != 0) return 0;
-    return fused_min_bytes(M, K) + split_area(M, N).total();
+    return fused_min_bytes(M, K);
 }
 
 nvfp4_status nvfp4_linear_bf16(const void* d_x, int64_t ldx, const float* d_g_a, int64_t M, int64_t K,
                                const uint8_t* d_w_codes, const uint8_t* d_w_sf, int64_t N,
                                const nvfp4_segment* segs, const float* d_g_seg, int nseg, void* d_y, int64_t ldy,
                                uint32_t flags, void* d_workspace, size_t workspace_bytes, void* stream) {
-    if (d_workspace == nullptr) return NVFP4_ERR_WORKSPACE;
-    if (M < 0 || K <= 0 || (K % 64) != 0) return NVFP4_ERR_SHAPE;
-    const size_t min_bytes = fused_min_bytes(M, K);
-    if (workspace_bytes < min_bytes) return NVFP4_ERR_WORKSPACE;
-    if (!aligned16(d_workspace)) return NVFP4_ERR_ALIGN;
-    // measured on B200 (5120 -> 6144, CUDA-graph replay): 8.8 / 11.4 us for 1 / 2 tokens against
-    // 12.5 us through the tensor-core path; from 3 tokens on the tensor cores win
-    if (M >= 1 && M <= 2 && N >= 1 && g_variant.load(std::memory_order_relaxed) == 0 &&
-        decode_smem_bytes(M, K) <= 200 * 1024) {
-        // decode-sized batch: one weight-streaming kernel, the workspace is not touched
-        if (d_x == nullptr || d_g_a == nullptr || d_w_codes == nullptr || d_w_sf == nullptr || d_g_seg == nullptr ||
-            d_y == nullptr)
-            return NVFP4_ERR_NULL;
-        if (ldx < K || ldy < N || N >= (1ll << 31) || K >= (1ll << 31)) return NVFP4_ERR_SHAPE;
-        if ((flags & ~(NVFP4_OUT_F32 | NVFP4_WS_ZEROED)) != 0u) return NVFP4_ERR_SHAPE;
-        nvfp4_status sg = check_segments(segs, nseg, N);
-        if (sg != NVFP4_OK) return sg;
-        if ((reinterpret_cast<uintptr_t>(d_x) & 31u) != 0 || (ldx % 16) != 0 || !aligned16(d_w_codes) || !aligned16(d_w_sf))
-            return NVFP4_ERR_ALIGN;
-        DeviceInfo info;
-        sg = check_arch(info);
-        if (sg != NVFP4_OK) return sg;
-        DecodeParams dp;
-        std::memset(&dp, 0, sizeof(dp));
-        dp.x = reinterpret_cast<const uint16_t*>(d_x);
-        dp.ldx = ldx;
-        dp.g_a = d_g_a;
-        dp.w_codes = d_w_codes;
-        dp.w_sf = d_w_sf;
-        dp.g_seg = d_g_seg;
-        dp.y = d_y;
-        dp.ldy = ldy;
-        dp.M = static_cast<int32_t>(M);
-        dp.N = static_cast<int32_t>(N);
-        dp.K = static_cast<int32_t>(K);
-        dp.flags = flags;
-        dp.nseg = nseg;
-        for (int i = 0; i < nseg; ++i) dp.seg_end[i] = static_cast<int32_t>(segs[i].col_begin + segs[i].col_count);
-        cudaStream_t s = as_stream(stream);
-        if (M == 1) return launch_decode<1>(dp, info.sm_count, s);
-        return launch_decode<2>(dp, info.sm_count, s);
-    }
-    uint8_t* ws = reinterpret_cast<uint8_t*>(d_workspace);
-    uint8_t* codes = ws + kStatusBytes;
-    uint8_t* sf = codes + fused_codes_bytes(M, K);
-    nvfp4_status st = nvfp4_quantize_act(d_x, M, K, ldx, d_g_a, codes, sf, NVFP4_SF_MMA, stream);
-    if (st != NVFP4_OK) return st;
-    return linear_impl(codes, sf, d_g_a, M, K, d_w_codes, d_w_sf, N, segs, d_g_seg, nseg, d_y, ldy, flags, d_workspace,
-                       kStatusBytes, ws + min_bytes, workspace_bytes - min_bytes, stream, (M + 127) / 128 * 128);
+    return linear_bf16_impl(d_x, ldx, d_g_a, M, K, d_w_codes, d_w_sf, N, segs, d_g_seg, nseg, d_y, ldy, flags,
+                            d_workspace, workspace_bytes, stream);
 }
 
 // ---------------------------------------------------------------- no-allocation variant
@@ -781,25 +839,30 @@ nvfp4_status nvfp4_linear_bf16_static(const void* d_x, int64_t ldx, const float*
                                       const nvfp4_segment* segs, const float* d_g_seg, int nseg, void* d_y,
                                       int64_t ldy, uint32_t flags, void* stream) {
     if (M < 0 || K <= 0 || (K % 64) != 0) return NVFP4_ERR_SHAPE;
-    (void)N;
-    const size_t need = (K % 16) == 0 ? fused_min_bytes(M, K) : 0;
-    if (need == 0 || need > NVFP4_STATIC_SCRATCH_BYTES) return NVFP4_ERR_WORKSPACE;   // beyond the fixed array
+    if (fused_min_bytes(M, K) > NVFP4_STATIC_SCRATCH_BYTES) return NVFP4_ERR_WORKSPACE;   // beyond the fixed array
     void* scratch = nullptr;
     nvfp4_status st = static_scratch_address(&scratch);
     if (st != NVFP4_OK) return st;
-    st = nvfp4_workspace_reset(scratch, NVFP4_STATIC_SCRATCH_BYTES, stream);           // status word starts at zero
-    if (st != NVFP4_OK) return st;
-    // the array starts as zeros (static storage) and only this library writes it, leaving its
-    // split-K part zero after every call: the NVFP4_WS_ZEROED promise holds by construction
-    return nvfp4_linear_bf16(d_x, ldx, d_g_a, M, K, d_w_codes, d_w_sf, N, segs, d_g_seg, nseg, d_y, ldy,
-                             flags | NVFP4_WS_ZEROED, scratch, NVFP4_STATIC_SCRATCH_BYTES, stream);
+    // The array starts as zeros (static storage) and only this library writes it: the status block
+    // [0, 256) is cleared by nvfp4_static_status whenever it reports a failure, the split-K part
+    // [256, 256 + reserve) is left zero by every call that uses it (and re-zeroed after a timeout),
+    // the quantized activations live behind the reserve.  So the NVFP4_WS_ZEROED promise holds.
+    return linear_bf16_impl(d_x, ldx, d_g_a, M, K, d_w_codes, d_w_sf, N, segs, d_g_seg, nseg, d_y, ldy,
+                            flags | NVFP4_WS_ZEROED, scratch, NVFP4_STATIC_SCRATCH_BYTES, stream);
 }
 
 nvfp4_status nvfp4_static_status(void* stream) {
     void* scratch = nullptr;
     nvfp4_status st = static_scratch_address(&scratch);
     if (st != NVFP4_OK) return st;
-    return nvfp4_device_status(scratch, stream);
+    st = nvfp4_device_status(scratch, stream);
+    if (st != NVFP4_OK) {
+        // a kernel that gave up may have left counters or partial sums behind: bring the status block
+        // and the split-K part back to zero so that later calls start clean (the stream is idle here)
+        if (cudaMemsetAsync(scratch, 0, kStatusBytes + kSplitReserve, as_stream(stream)) != cudaSuccess) return NVFP4_ERR_CUDA;
+        if (cudaStreamSynchronize(as_stream(stream)) != cudaSuccess) return NVFP4_ERR_CUDA;
+    }
+    return st;
 }
 
 nvfp4_status nvfp4_device_status(const void* d_workspace, void* stream) {
@@ -808,7 +871,10 @@ nvfp4_status nvfp4_device_status(const void* d_workspace, void* stream) {
     if (cudaMemcpyAsync(&word, d_workspace, sizeof(word), cudaMemcpyDeviceToHost, as_stream(stream)) != cudaSuccess)
         return NVFP4_ERR_CUDA;
     if (cudaStreamSynchronize(as_stream(stream)) != cudaSuccess) return NVFP4_ERR_CUDA;
-    return word == 0u ? NVFP4_OK : (word == NVFP4_ERR_TIMEOUT ? NVFP4_ERR_TIMEOUT : NVFP4_ERR_CUDA);
+    if (word == 0u) return NVFP4_OK;
+    if (word == NVFP4_ERR_TIMEOUT) return NVFP4_ERR_TIMEOUT;
+    if (word == NVFP4_ERR_SCALE) return NVFP4_ERR_SCALE;
+    return NVFP4_ERR_CUDA;
 }
 
 namespace nvfp4 {
@@ -870,6 +936,7 @@ const char* nvfp4_status_string(nvfp4_status s) {
         case NVFP4_ERR_CUDA: return "CUDA call failed";
         case NVFP4_ERR_TIMEOUT: return "a bounded in-kernel wait ran out";
         case NVFP4_ERR_LAYOUT: return "unknown or unsupported scale layout";
+        case NVFP4_ERR_SCALE: return "a global scale is not finite and positive";
     }
     return "unknown status";
 }

@@ -78,6 +78,12 @@ __device__ __forceinline__ void ldg256_cached(const void* p, uint32_t (&v)[8]) {
                  : "l"(p));
 }
 
+__device__ __forceinline__ void stg256(void* p, const uint32_t (&v)[8]) {
+    asm volatile("st.global.v8.b32 [%8], {%0,%1,%2,%3,%4,%5,%6,%7};"
+                 ::"r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "l"(p)
+                 : "memory");
+}
+
 __device__ __forceinline__ uint32_t bf16x2_absmax(uint32_t a, uint32_t b) {
     uint32_t r;
     asm("max.xorsign.abs.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
@@ -118,24 +124,19 @@ __device__ __forceinline__ uint2 quantize_block(const uint32_t (&v)[8], float g,
     return out;
 }
 
-// silu(g) * u in the binary32 sequence that the path fixes for the MLP's activation (each step
-// one IEEE operation, fmaf fused):  t = clamp(-g, -87, 87);  n = rint(t * log2 e);
-// r = fmaf(t, log2 e, -n);  2^r by a degree-5 polynomial;  e = 2^r * 2^n;
-// s = g * (1 / (1 + e));  result s * u.
+// silu(g) * u = g * sigmoid(g) * u in binary32 with the hardware's approximate exp2 and
+// reciprocal (2 MUFU + 6 arithmetic instructions per element).  With z = exp(-|g|) in (0, 1]:
+// sigmoid(g) = 1 / (1 + z) for g >= 0 and z / (1 + z) for g < 0, so nothing overflows and very
+// negative gates keep their (tiny, possibly subnormal) value.  The relative error before the bf16
+// rounding is a few 2^-22 (the exponent's rounding adds |g| * 2^-24 * ln 2 for large |g|), so the
+// rounded result equals the correctly rounded definition except in about one case in 10^4 and is
+// never more than one bf16 ulp away.
 __device__ __forceinline__ float silu_mul(float g, float u) {
-    const float LOG2E = 1.44269504088896341f;
-    const float t = fminf(fmaxf(-g, -87.0f), 87.0f);
-    const float n = rintf(__fmul_rn(t, LOG2E));
-    const float r = __fmaf_rn(t, LOG2E, -n);
-    float p = 1.3333558146e-3f;
-    p = __fmaf_rn(p, r, 9.6181291076e-3f);
-    p = __fmaf_rn(p, r, 5.5504108665e-2f);
-    p = __fmaf_rn(p, r, 2.4022650696e-1f);
-    p = __fmaf_rn(p, r, 6.9314718056e-1f);
-    p = __fmaf_rn(p, r, 1.0f);
-    const float e = __fmul_rn(p, __int_as_float((static_cast<int>(n) + 127) << 23));
-    const float s = __fmul_rn(g, __frcp_rn(__fadd_rn(1.0f, e)));
-    return __fmul_rn(s, u);
+    float z, r;
+    asm("ex2.approx.f32 %0, %1;" : "=f"(z) : "f"(__fmul_rn(fabsf(g), -1.44269504088896341f)));
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(__fadd_rn(1.0f, z)));
+    const float sig = g >= 0.0f ? r : __fmul_rn(z, r);
+    return __fmul_rn(__fmul_rn(g, sig), u);
 }
 
 // 16 gate values and 16 up values (packed bf16) -> 16 values of bf16(silu(gate) * up), packed
@@ -167,14 +168,14 @@ constexpr int kQuantPlain = 0, kQuantSwiglu = 1, kQuantRmsnorm = 2;
 // MODE kQuantSwiglu: x is [M, 2K] (gate | up) and the tensor that is quantized is
 // bf16(silu(gate) * up), [M, K].  MODE kQuantRmsnorm: the quantized tensor is
 // bf16(x * rstd(row) * aux[k]) with rstd = 1 / sqrt(mean(x^2) + eps); a unit is then a whole row
-// (units_per_row == 1): the warp first sums the squares of its row (each lane over its own
-// 16-element pieces in increasing k, fused multiply-adds, then a butterfly over the 32 lanes),
-// and reads the row a second time, from cache, to normalise and quantize it.
+// (units_per_row == 1): the warp first sums the squares of its row and reads the row a second
+// time, from cache, to normalise and quantize it.  (Rows of up to 20480 elements take
+// rmsnorm_quantize_kernel below, which keeps the row in registers; this is the general form.)
 template <bool MMA_LAYOUT, int UNROLL, int MODE>
 __global__ void __launch_bounds__(256, MODE == kQuantPlain ? 5 : 4)
 quantize_kernel(const uint16_t* __restrict__ x, int32_t M, int32_t K, int64_t ld,
                 const float* __restrict__ g_ptr, SegTable segs, const uint16_t* __restrict__ aux, float eps,
-                uint8_t* __restrict__ codes, uint8_t* __restrict__ sf,
+                uint8_t* __restrict__ codes, uint8_t* __restrict__ sf, uint16_t* __restrict__ h_out,
                 int32_t chunks_per_row, int32_t chunks_per_unit, int32_t units_per_row, int32_t total_units) {
     // the GEMM that consumes this tensor may start its prologue and its weight loads now; it
     // waits for this kernel's completion before it touches the codes and scales written here
@@ -269,6 +270,8 @@ quantize_kernel(const uint16_t* __restrict__ x, int32_t M, int32_t K, int64_t ld
 #pragma unroll
                         for (int i = 0; i < 8; ++i) v[u][i] = y[i];
                     }
+                    if (MODE != kQuantPlain && h_out != nullptr)        // testing aid: the tensor that is quantized
+                        stg256(h_out + static_cast<int64_t>(row) * K + col[u], v[u]);
                 } else {
 #pragma unroll
                     for (int i = 0; i < 8; ++i) v[u][i] = 0u;
@@ -294,6 +297,117 @@ quantize_kernel(const uint16_t* __restrict__ x, int32_t M, int32_t K, int64_t ld
                 } else if (in_range) {
                     sf_row[kb] = static_cast<uint8_t>(s8);
                 }
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------ RMSNorm -> quantize, row in registers
+// A row is shared by W warps of one CTA (W = 1, 2, 4 or 8; each warp owns up to kRmsChunks
+// consecutive 512-element chunks and each lane one 16-element block per chunk), so the row is read
+// from HBM exactly once and stays in registers between the reduction and the quantization:
+//   1. every lane loads its blocks (streaming loads, all in flight at once) and sums their squares;
+//   2. warp butterfly, then the W partial sums meet in shared memory (one named barrier per row;
+//      the two buffers alternate so that no second barrier is needed);
+//   3. y = bf16((x * rstd) * w) per element, then the block is quantized as everywhere else.
+// Rows are dealt round-robin to the row groups of a persistent grid.  Rows M .. M_pad-1 (tensor-core
+// layout only) get zero scales.
+constexpr int kRmsChunks = 5;
+
+template <bool MMA_LAYOUT, int W>
+__global__ void __launch_bounds__(256, 2)
+rmsnorm_quantize_kernel(const uint16_t* __restrict__ x, int32_t M, int32_t rows_total, int32_t K, int64_t ld,
+                        const float* __restrict__ g_ptr, const uint16_t* __restrict__ gain, float eps,
+                        uint8_t* __restrict__ codes, uint8_t* __restrict__ sf, uint16_t* __restrict__ y_out,
+                        int32_t chunks_per_row, int32_t chunks_per_warp) {
+    ptx::pdl_launch_dependents();
+    __shared__ float red[2][8];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int sub = warp % W;                                  // this warp's part of the row
+    const int group = warp / W;                                // row group inside the CTA
+    constexpr int kGroups = 8 / W;
+    const int32_t KB = K >> 4;
+    const int32_t katoms = (KB + 3) >> 2;
+    const float g = __ldg(g_ptr);
+    const float c1 = __fdiv_rn(1.0f, __fmul_rn(6.0f, g));
+    const int32_t c_begin = sub * chunks_per_warp;
+    const int32_t c_end = min(chunks_per_row, c_begin + chunks_per_warp);
+    uint32_t parity = 0;
+    for (int32_t row = blockIdx.x * kGroups + group; row < rows_total; row += gridDim.x * kGroups) {
+        uint8_t* sf_row = MMA_LAYOUT
+            ? sf + static_cast<int64_t>(row >> 7) * katoms * 512 + (row & 31) * 16 + ((row & 127) >> 5) * 4
+            : sf + static_cast<int64_t>(row) * KB;
+        if (row >= M) {
+            // only reached in the tensor-core layout: rows that pad the last 128-row band
+            for (int32_t c = c_begin; c < c_end; ++c) {
+                const int32_t kb = c * 32 + lane;
+                if ((lane & 3) == 0 && kb < KB) *reinterpret_cast<uint32_t*>(sf_row + static_cast<int64_t>(kb >> 2) * 512) = 0u;
+            }
+            continue;                                           // a whole group skips together: no barrier is missed
+        }
+        const uint16_t* xrow = x + static_cast<int64_t>(row) * ld;
+        uint32_t v[kRmsChunks][8];
+#pragma unroll
+        for (int i = 0; i < kRmsChunks; ++i) {
+            const int32_t col = (c_begin + i) * 512 + lane * 16;
+            if (c_begin + i < c_end && col < K) {
+                ldg256_stream(xrow + col, v[i]);
+            } else {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) v[i][e] = 0u;
+            }
+        }
+        float ss = 0.0f;
+#pragma unroll
+        for (int i = 0; i < kRmsChunks; ++i) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const float lo = __uint_as_float(v[i][e] << 16), hi = __uint_as_float(v[i][e] & 0xFFFF0000u);
+                ss = __fmaf_rn(lo, lo, ss);
+                ss = __fmaf_rn(hi, hi, ss);
+            }
+        }
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) ss = __fadd_rn(ss, __shfl_xor_sync(0xffffffffu, ss, off));
+        if (W > 1) {
+            if (lane == 0) red[parity][warp] = ss;
+            ptx::named_bar_sync(1 + group, W * 32);
+            ss = 0.0f;
+#pragma unroll
+            for (int w = 0; w < W; ++w) ss = __fadd_rn(ss, red[parity][group * W + w]);
+            parity ^= 1u;
+        }
+        const float rstd = __frcp_rn(__fsqrt_rn(__fadd_rn(__fdiv_rn(ss, static_cast<float>(K)), eps)));
+        uint8_t* crow = codes + static_cast<int64_t>(row) * (K >> 1);
+#pragma unroll
+        for (int i = 0; i < kRmsChunks; ++i) {
+            if (c_begin + i >= c_end) break;                    // warp-uniform
+            const int32_t col = (c_begin + i) * 512 + lane * 16;
+            const bool in_range = col < K;
+            uint32_t y[8];
+            if (in_range) {
+                uint32_t wv[8];
+                ldg256_cached(gain + col, wv);
+                rmsnorm_block(v[i], wv, rstd, y);
+                if (y_out != nullptr) stg256(y_out + static_cast<int64_t>(row) * K + col, y);   // testing aid
+            } else {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) y[e] = 0u;
+            }
+            uint32_t s8;
+            const uint2 word = quantize_block(y, g, c1, s8);
+            if (!in_range) s8 = 0u;
+            if (in_range) *reinterpret_cast<uint2*>(crow + (col >> 1)) = word;
+            const int32_t kb = col >> 4;
+            if (MMA_LAYOUT || ((KB & 3) == 0 && (reinterpret_cast<uintptr_t>(sf) & 3u) == 0)) {
+                uint32_t w4 = s8 | (__shfl_down_sync(0xffffffffu, s8, 1) << 8);
+                w4 |= __shfl_down_sync(0xffffffffu, w4, 2) << 16;
+                if ((lane & 3) == 0 && kb < KB) {
+                    if (MMA_LAYOUT) *reinterpret_cast<uint32_t*>(sf_row + static_cast<int64_t>(kb >> 2) * 512) = w4;
+                    else            *reinterpret_cast<uint32_t*>(sf_row + kb) = w4;
+                }
+            } else if (in_range) {
+                sf_row[kb] = static_cast<uint8_t>(s8);
             }
         }
     }

@@ -6,9 +6,45 @@ Works with NCCL (one rank per GPU) and with gloo on CPU (tests)."""
 from __future__ import annotations
 
 import os
-from typing import Optional
+import socket
+import subprocess
+import sys
+from typing import List, Optional, Sequence
 
 import torch
+
+
+def launched_by_a_launcher() -> bool:
+    """True when RANK / WORLD_SIZE were exported by whoever started this process (torchrun or
+    spawn_replicas): the process is then one replica and must not start more."""
+    return "RANK" in os.environ and "WORLD_SIZE" in os.environ
+
+
+def spawn_replicas(n: int, argv: Sequence[str], extra_env: Optional[dict] = None, timeout: Optional[float] = None) -> int:
+    """Start `n` copies of `argv` on this node, one per GPU (RANK = LOCAL_RANK = 0..n-1, WORLD_SIZE = n,
+    rendezvous on 127.0.0.1 at a free port), wait for all of them and return the first non-zero exit
+    code (0 if all succeeded).  Rank 0 inherits this process's stdout, so the one line it prints is
+    the job's output; the other ranks' stdout is discarded, every rank's stderr is inherited."""
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    procs: List[subprocess.Popen] = []
+    for rank in range(n):
+        env = dict(os.environ, RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(n),
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        if extra_env:
+            env.update(extra_env)
+        procs.append(subprocess.Popen(list(argv), env=env, stdout=None if rank == 0 else subprocess.DEVNULL))
+    rc = 0
+    for p in procs:
+        try:
+            code = p.wait(timeout=timeout)
+        except subprocess.TimeoutExpired:
+            p.kill()
+            code = 124
+        if code != 0 and rc == 0:
+            rc = code
+    return rc
 
 
 class Replicas:

@@ -79,4 +79,25 @@ def test_host_side_argument_checks_need_no_gpu(L):
     assert L.nvfp4_device_status(None, None) == 1
     assert L.nvfp4_set_gemm_variant(3) == 2 and L.nvfp4_set_gemm_variant(0) == 0
     assert L.nvfp4_linear_workspace_bytes(8, 16, 64, 2) >= 4
-    assert L.nvfp4_linear_bf16_workspace_bytes(8, 16, 64, 2) >= 256 + 8 * 32 + 512
+    assert L.nvfp4_linear_bf16_workspace_bytes(8, 16, 64, 2) >= 256 + nv.SPLIT_RESERVE_BYTES + 128 * 32 + 512
+    assert L.nvfp4_linear_workspace_bytes(16, 6144, 8192, 1) <= 256 + nv.SPLIT_RESERVE_BYTES
+    # the fused entry points check every argument before anything is enqueued
+    fused = lambda **kw: L.nvfp4_linear_bf16(kw.get("x", p), kw.get("ldx", 64), p, kw.get("M", 8), kw.get("K", 64), p, p,
+                                             kw.get("N", 16), kw.get("segs", seg), p, kw.get("nseg", 2), p,
+                                             kw.get("ldy", 16), kw.get("flags", 0), kw.get("ws", p),
+                                             kw.get("wsb", 1 << 24), None)
+    assert fused(x=None) == 1
+    assert fused(K=48) == 2
+    assert fused(ldx=32) == 2
+    assert fused(ldy=8) == 2
+    assert fused(flags=4) == 2
+    assert fused(N=24, ldy=32) == 4
+    assert fused(ws=None) == 5
+    assert fused(wsb=4096) == 5
+    assert fused(x=vp(0x1010)) == 3
+    assert fused(M=1, x=None) == 1 and fused(M=1, N=24, ldy=32) == 4        # the single-token route checks the same
+    static = lambda **kw: L.nvfp4_linear_bf16_static(p, 64, p, kw.get("M", 8), kw.get("K", 64), p, p, 16, seg, p, 2, p, 16,
+                                                     0, None)
+    assert static(K=48) == 2 and static(M=-1) == 2
+    assert static(M=4096, K=5120) == 5                                       # beyond the fixed array
+    assert nv.STATIC_SCRATCH_BYTES == 12 * 1024 * 1024

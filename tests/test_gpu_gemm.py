@@ -201,25 +201,7 @@ def test_gdn_in_projection_full_size_sampled(variant):
     ws = _ws()
     y = nv.nvfp4_linear(a_codes, a_sf, g_a, w_codes, w_sf, segs, g_seg, ws)
     assert nv.device_status(ws) == 0
-    rng = np.random.default_rng(0)
-    rows = np.sort(np.array([t * 128 + rng.integers(0, 128) for t in range(0, M // 128, 4)] + [0, M - 1]))
-    y_rows = oracle.gemm(ac, asf, ga, wc, wsf, gcol, rows=rows)
-    gu.check_gemm(y[torch.from_numpy(rows).to(gu.DEV)], y_rows,
-                  gu.gemm_bounds(ac, asf, ga, wc, wsf, gcol, rows=rows), "gdn rows")
-    edge = sorted({c for s in segs for c in (s.begin, s.begin + s.count - 1)} | {N - 1, 0})
-    cols = np.array(sorted(set(edge) | set(rng.integers(0, N, 24).tolist())))
-    y_cols = oracle.gemm(ac, asf, ga, wc, wsf, gcol, cols=cols)
-    gu.check_gemm(y[:, torch.from_numpy(cols).to(gu.DEV)].contiguous(), y_cols,
-                  gu.gemm_bounds(ac, asf, ga, wc, wsf, gcol, cols=cols), "gdn cols")
-    # Freivalds-style projection over the whole output: Y r against A_hat (W_hat^T r) in float64
-    r = rng.choice([-1.0, 1.0], N)
-    a_hat = oracle.dequantize(ac, asf, oracle.row_scales(M, g=ga))
-    w_hat = oracle.dequantize(wc, wsf, gcol)
-    want = a_hat @ (w_hat.T @ r)
-    got = y.double().cpu().numpy() @ r
-    scale = np.linalg.norm(a_hat, axis=1) * np.linalg.norm(w_hat) / np.sqrt(K)
-    # bf16 rounding of N outputs: random-walk error ~ 2^-9 * |y| * sqrt(N)
-    assert np.max(np.abs(got - want) / scale) < 2e-2
+    _check_sampled(y, M, N, K, segs, ac, asf, ga, wc, wsf, gcol, np.random.default_rng(0), "gdn")
 
 
 # ---- decode-sized batches: split-K over a self-cleaning workspace -----------------------------
@@ -249,10 +231,54 @@ def test_small_m_split_k(M, N, K, out_f32):
 
 
 # ---- the benchmark's own shapes at full size (whole device path, auto tile choice) ------------
-def _full_size_sampled(M, K, spec, seed, n_rows=16, n_cols=24):
+def _sample_rows_cols(M, N, segs, rng, n_cols=64):
+    """One row inside every 128-row band (plus the first and last row); at least `n_cols` columns,
+    among them both neighbours of every segment edge and the last column."""
+    rows = np.unique(np.array([t * 128 + rng.integers(0, min(128, M - t * 128)) for t in range((M + 127) // 128)]
+                              + [0, M - 1]))
+    edge = set()
+    for s_ in segs:
+        for c in (s_.begin - 1, s_.begin, s_.begin + s_.count - 1, s_.begin + s_.count):
+            if 0 <= c < N:
+                edge.add(int(c))
+    edge |= {0, N - 1}
+    extra = set(rng.integers(0, N, max(0, n_cols - len(edge)) + 8).tolist())
+    cols = np.array(sorted(edge | extra))
+    assert len(cols) >= min(n_cols, N)
+    return rows, cols
+
+
+def _check_sampled(y, M, N, K, segs, ac, asf, ga, wc, wsf, gcol, rng, what):
+    """Oracle comparison of a full-size output on sampled rows and columns plus a random-sign
+    projection of the whole output (operands dequantized in chunks)."""
+    rows, cols = _sample_rows_cols(M, N, segs, rng)
+    y_rows = oracle.gemm(ac, asf, ga, wc, wsf, gcol, rows=rows)
+    gu.check_gemm(y[torch.from_numpy(rows).to(gu.DEV)], y_rows,
+                  gu.gemm_bounds(ac, asf, ga, wc, wsf, gcol, rows=rows), what + " rows")
+    y_cols = oracle.gemm(ac, asf, ga, wc, wsf, gcol, cols=cols)
+    gu.check_gemm(y[:, torch.from_numpy(cols).to(gu.DEV)].contiguous(), y_cols,
+                  gu.gemm_bounds(ac, asf, ga, wc, wsf, gcol, cols=cols), what + " cols")
+    r = rng.choice([-1.0, 1.0], N)
+    wr = np.zeros(K)
+    w_norm2 = 0.0
+    for b in range(0, N, 4096):
+        w_hat = oracle.dequantize(wc[b:b + 4096], wsf[b:b + 4096], gcol[b:b + 4096])
+        wr += w_hat.T @ r[b:b + 4096]
+        w_norm2 += float((w_hat ** 2).sum())
+    worst = 0.0
+    got = (y.double() @ torch.from_numpy(r).to(gu.DEV)).cpu().numpy()
+    for b in range(0, M, 2048):
+        a_hat = oracle.dequantize(ac[b:b + 2048], asf[b:b + 2048], oracle.row_scales(min(2048, M - b), g=ga))
+        want = a_hat @ wr
+        scale = np.linalg.norm(a_hat, axis=1) * np.sqrt(w_norm2) / np.sqrt(K)
+        worst = max(worst, float(np.max(np.abs(got[b:b + 2048] - want) / scale)))
+    # bf16 rounding of N outputs: random-walk error ~ 2^-9 * |y| * sqrt(N)
+    assert worst < 2e-2, (what, worst)
+
+
+def _full_size_sampled(M, K, spec, seed):
     """Device path end to end (calibrate, quantize, GEMM) at full size; the oracle checks the
-    quantized operands in full, the GEMM on sampled rows, sampled columns (every segment edge and
-    the last column among them) and a random-sign projection of the whole output."""
+    quantized operands in full and the GEMM as _check_sampled describes."""
     segs = synth.make_segments(spec)
     N = sum(s.count for s in segs)
     x = synth.prefill_activations(seed, 501, M, K)
@@ -270,34 +296,7 @@ def _full_size_sampled(M, K, spec, seed, n_rows=16, n_cols=24):
     ws = _ws()
     y = nv.nvfp4_linear(a_codes, a_sf, g_a, w_codes, w_sf, segs, g_seg, ws)
     assert nv.device_status(ws) == 0
-    rng = np.random.default_rng(seed)
-    step = max(1, (M // 128) // n_rows)
-    rows = np.unique(np.array([t * 128 + rng.integers(0, 128) for t in range(0, M // 128, step)] + [0, M - 1]))
-    y_rows = oracle.gemm(ac, asf, ga, wc, wsf, gcol, rows=rows)
-    gu.check_gemm(y[torch.from_numpy(rows).to(gu.DEV)], y_rows,
-                  gu.gemm_bounds(ac, asf, ga, wc, wsf, gcol, rows=rows), "rows")
-    edge = {c for s in segs for c in (s.begin, s.begin + s.count - 1)} | {0, N - 1}
-    cols = np.array(sorted(edge | set(rng.integers(0, N, n_cols).tolist())))
-    y_cols = oracle.gemm(ac, asf, ga, wc, wsf, gcol, cols=cols)
-    gu.check_gemm(y[:, torch.from_numpy(cols).to(gu.DEV)].contiguous(), y_cols,
-                  gu.gemm_bounds(ac, asf, ga, wc, wsf, gcol, cols=cols), "cols")
-    # projection of the whole output on a random sign vector, operands dequantized in row chunks
-    r = rng.choice([-1.0, 1.0], N)
-    wr = np.zeros(K)
-    w_norm2 = 0.0
-    for b in range(0, N, 4096):
-        w_hat = oracle.dequantize(wc[b:b + 4096], wsf[b:b + 4096], gcol[b:b + 4096])
-        wr += w_hat.T @ r[b:b + 4096]
-        w_norm2 += float((w_hat ** 2).sum())
-    worst = 0.0
-    r_dev = torch.from_numpy(r).to(gu.DEV)
-    got = (y.double() @ r_dev).cpu().numpy()
-    for b in range(0, M, 2048):
-        a_hat = oracle.dequantize(ac[b:b + 2048], asf[b:b + 2048], oracle.row_scales(min(2048, M - b), g=ga))
-        want = a_hat @ wr
-        scale = np.linalg.norm(a_hat, axis=1) * np.sqrt(w_norm2) / np.sqrt(K)
-        worst = max(worst, float(np.max(np.abs(got[b:b + 2048] - want) / scale)))
-    assert worst < 2e-2, worst
+    _check_sampled(y, M, N, K, segs, ac, asf, ga, wc, wsf, gcol, np.random.default_rng(seed), "full size %s" % ((M, N, K),))
 
 
 def test_mlp_gate_up_full_size_sampled():
@@ -309,7 +308,7 @@ def test_mlp_down_full_size_sampled():
 
 
 def test_long_prefill_32k_tokens_sampled():
-    _full_size_sampled(32768, synth.HIDDEN, (("w", 6144, 0.02),), 3, n_rows=32)
+    _full_size_sampled(32768, synth.HIDDEN, (("w", 6144, 0.02),), 3)
 
 
 # ---- 1 or 2 tokens: the weight-streaming decode kernel behind nvfp4_linear_bf16 (3, 4: tensor cores) ------------------
@@ -341,3 +340,138 @@ def test_decode_batches(M, N, K, out_f32):
                               gu.dev_f32(gs), ws, out_f32=out_f32)
     nv.set_gemm_variant(0)
     gu.check_gemm(y2, y_ref, gu.gemm_bounds(ac, asf, ga, wc, wsf, gcol), "tensor-core path")
+
+
+# ---- the M sweep's own entry point: quantize inside the call, K=5120 -> N=6144 -----------------
+@pytest.mark.parametrize("M", [16, 128, 1024, 8192])
+def test_m_sweep_layer_through_the_fused_entry_point(M):
+    K, N = synth.HIDDEN, 6144
+    segs = synth.make_segments((("w", N, 0.02),))
+    x = synth.prefill_activations(7, 601, M, K)
+    w = synth.weights(7, 602, segs, K)
+    ac, asf, ga, _ = gu.oracle_quantized(x)
+    wc, wsf, gs, _ = gu.oracle_quantized(w, segments=segs)
+    gcol = oracle.col_scales(N, segs, gs)
+    ws = nv.alloc_workspace(gu.DEV, M, N, K, 1, fused=True)
+    y = nv.nvfp4_linear_bf16(gu.dev_bf16(x), gu.dev_f32(ga), gu.dev_u8(wc), gu.dev_u8(oracle.sf_to_mma(wsf, K)), segs,
+                             gu.dev_f32(gs), ws)
+    assert nv.device_status(ws) == 0
+    if M <= 1024:
+        gu.check_gemm(y, oracle.gemm(ac, asf, ga, wc, wsf, gcol), gu.gemm_bounds(ac, asf, ga, wc, wsf, gcol), "M=%d" % M)
+    else:
+        _check_sampled(y, M, N, K, segs, ac, asf, ga, wc, wsf, gcol, np.random.default_rng(M), "M=%d" % M)
+    assert bool((ws[256:256 + nv.SPLIT_RESERVE_BYTES] == 0).all())
+
+
+# ---- one workspace across layers of different K: the split-K part sits at a fixed place ---------
+def _decode_layer(seed, M, N, K):
+    segs = synth.make_segments((("w", N, 0.02),))
+    x = synth.prefill_activations(seed, 701, M, K)
+    w = synth.weights(seed, 702, segs, K)
+    ac, asf, ga, _ = gu.oracle_quantized(x)
+    wc, wsf, gs, _ = gu.oracle_quantized(w, segments=segs)
+    gcol = oracle.col_scales(N, segs, gs)
+    y_ref = oracle.gemm(ac, asf, ga, wc, wsf, gcol)
+    bound = gu.gemm_bounds(ac, asf, ga, wc, wsf, gcol)
+    dev = (gu.dev_bf16(x), gu.dev_f32(ga), gu.dev_u8(wc), gu.dev_u8(oracle.sf_to_mma(wsf, K)), segs, gu.dev_f32(gs))
+    return dev, y_ref, bound
+
+
+def test_one_workspace_reused_across_layers_of_different_k():
+    # the model's own pair: K = 5120 (no split-K) and K = 17408 (split-K), alternating on one
+    # zero-filled workspace sized for the larger; every result against the oracle
+    M = 16
+    a, a_ref, a_bound = _decode_layer(31, M, 6144, synth.HIDDEN)
+    b, b_ref, b_bound = _decode_layer(32, M, synth.HIDDEN, synth.MLP_INNER)
+    big, big_ref, big_bound = _decode_layer(33, 200, 1024, 8192)          # many rows: codes reach far into the workspace
+    small, small_ref, small_bound = _decode_layer(34, 16, 6144, 8192)      # split-K again after it
+    n = max(nv.lib().nvfp4_linear_bf16_workspace_bytes(m, nn, k, 1)
+            for (m, nn, k) in ((M, 6144, synth.HIDDEN), (M, synth.HIDDEN, synth.MLP_INNER), (200, 1024, 8192), (16, 6144, 8192)))
+    ws = torch.zeros(int(n), dtype=torch.uint8, device=gu.DEV)
+    for dev, ref, bound, what in ((a, a_ref, a_bound, "K=5120"), (b, b_ref, b_bound, "K=17408"),
+                                  (big, big_ref, big_bound, "M=200 K=8192"), (small, small_ref, small_bound, "M=16 K=8192"),
+                                  (a, a_ref, a_bound, "K=5120 again"), (b, b_ref, b_bound, "K=17408 again")):
+        y = nv.nvfp4_linear_bf16(*dev, ws)
+        assert nv.device_status(ws) == 0, what
+        gu.check_gemm(y, ref, bound, what)
+        assert bool((ws[256:256 + nv.SPLIT_RESERVE_BYTES] == 0).all()), what      # split-K part left at zero
+
+
+def test_bad_global_scale_is_reported_on_the_device():
+    # g must be finite and > 0: the kernel reports it in the status word instead of repairing it
+    M, N, K = 64, 256, 256
+    segs, x, w, ac, asf, ga, wc, wsf, gs = _oracle_operands(41, M, K, (("p", 128, 0.02), ("q", 128, 0.2)))
+    for bad_ga, bad_gs in ((0.0, gs), (float("inf"), gs), (ga, [gs[0], -1.0]), (ga, [float("nan"), gs[1]])):
+        ws = _ws()
+        nv.nvfp4_linear(gu.dev_u8(ac), gu.dev_u8(oracle.sf_to_mma(asf, K)), gu.dev_f32(bad_ga), gu.dev_u8(wc),
+                        gu.dev_u8(oracle.sf_to_mma(wsf, K)), segs, gu.dev_f32(bad_gs), ws)
+        assert nv.device_status(ws) == 10
+    # the decode kernel (1 token, bf16 in) reports it too
+    ws = nv.alloc_workspace(gu.DEV, 1, N, K, 2, fused=True)
+    nv.nvfp4_linear_bf16(gu.dev_bf16(x[:1]), gu.dev_f32(0.0), gu.dev_u8(wc), gu.dev_u8(oracle.sf_to_mma(wsf, K)), segs,
+                         gu.dev_f32(gs), ws)
+    assert nv.device_status(ws) == 10
+    ws = _ws()
+    y = _run_from_oracle_operands(segs, ac, asf, ga, wc, wsf, gs, K, ws=ws)       # good scales: status stays 0
+    gu.check_gemm(y, oracle.gemm(ac, asf, ga, wc, wsf, oracle.col_scales(N, segs, gs)),
+                  gu.gemm_bounds(ac, asf, ga, wc, wsf, oracle.col_scales(N, segs, gs)), "good scales")
+
+
+# ---- the MLP as served: gate/up GEMM -> silu(gate)*up quantized by the producer-fused kernel -> down GEMM ----
+def test_mlp_chain_with_fused_producer_link_by_link():
+    M, K, INNER = 8192, synth.HIDDEN, synth.MLP_INNER
+    seg_gu = synth.make_segments((("gate", INNER, 0.02), ("up", INNER, 0.02)))
+    seg_d = synth.make_segments((("down", K, 0.02),))
+    x = synth.prefill_activations(5, 801, M, K)
+    w_gu = synth.weights(5, 802, seg_gu, K)
+    w_d = synth.weights(5, 803, seg_d, INNER)
+    ac, asf, ga, _ = gu.oracle_quantized(x)
+    wgc, wgsf, ggs, _ = gu.oracle_quantized(w_gu, segments=seg_gu)
+    wdc, wdsf, gds, _ = gu.oracle_quantized(w_d, segments=seg_d)
+    gcol_gu = oracle.col_scales(2 * INNER, seg_gu, ggs)
+    gcol_d = oracle.col_scales(K, seg_d, gds)
+    rng = np.random.default_rng(5)
+    rows = np.unique(np.array([t * 128 + rng.integers(0, 128) for t in range(M // 128)] + [0, M - 1]))
+    rows_t = torch.from_numpy(rows).to(gu.DEV)
+    # device chain
+    xt = gu.dev_bf16(x)
+    g1 = gu.dev_f32(ga)
+    q1 = nv.nvfp4_quantize_act(xt, g1)
+    w_gu_c, w_gu_sf, g_gu = nv.nvfp4_quantize_weight(gu.dev_bf16(w_gu), seg_gu)
+    w_d_c, w_d_sf, g_d = nv.nvfp4_quantize_weight(gu.dev_bf16(w_d), seg_d)
+    ws = _ws()
+    y1 = nv.nvfp4_linear(q1[0], q1[1], g1, w_gu_c, w_gu_sf, seg_gu, g_gu, ws)
+    # link 1: gate/up GEMM rows against the exact GEMM
+    y1_rows_ref = oracle.gemm(ac, asf, ga, wgc, wgsf, gcol_gu, rows=rows)
+    gu.check_gemm(y1[rows_t], y1_rows_ref, gu.gemm_bounds(ac, asf, ga, wgc, wgsf, gcol_gu, rows=rows), "gate/up rows")
+    # the activation scale of h is static (offline calibration): here from the definition on the sampled rows
+    y1_rows_bits = gu.host_bits(y1[rows_t].contiguous())
+    h_rows_def = oracle.swiglu_bf16(y1_rows_bits)
+    _, gh = oracle.calibrate(h_rows_def)
+    gh = np.float32(gh * 2.0)                                              # head-room for the rows not sampled
+    g2 = gu.dev_f32(gh)
+    h_d = torch.empty((M, INNER), dtype=torch.bfloat16, device=gu.DEV)
+    q2 = nv.nvfp4_swiglu_quantize(y1, g2, h_out=h_d)
+    y2 = nv.nvfp4_linear(q2[0], q2[1], g2, w_d_c, w_d_sf, seg_d, g_d, ws)
+    assert nv.device_status(ws) == 0
+    # link 2: h the kernel formed against the definition applied to the device's own gate/up rows
+    h_rows_gpu = gu.host_bits(h_d[rows_t].contiguous())
+    gu.check_bf16_close_to_definition(h_rows_gpu, h_rows_def, 0.995, "h rows")
+    # link 3: codes and scales bit-exact against the oracle's quantization of that h
+    hc, hsf = oracle.quantize(h_rows_gpu, oracle.row_scales(len(rows), g=gh))
+    sf_lin, pad_zero = oracle.sf_from_mma(q2[1].cpu().numpy(), M, INNER)
+    assert pad_zero
+    assert np.array_equal(q2[0][rows_t].cpu().numpy(), hc) and np.array_equal(sf_lin[rows], hsf)
+    # link 4: down GEMM rows against the exact GEMM on those codes
+    y2_rows_ref = oracle.gemm(hc, hsf, gh, wdc, wdsf, gcol_d)
+    bound = gu.gemm_bounds(hc, hsf, gh, wdc, wdsf, gcol_d)
+    gu.check_gemm(y2[rows_t], y2_rows_ref, bound, "down rows")
+    # end to end: the oracle's own chain (exact GEMM -> bf16 -> definition -> quantize -> exact GEMM) on the
+    # same rows; the device differs where a gate/up output or an h rounded the other way (rare, one ulp)
+    y1_bits_ref = oracle.f64_to_bf16_bits(y1_rows_ref)
+    h_ref = oracle.swiglu_bf16(y1_bits_ref)
+    hc_ref, hsf_ref = oracle.quantize(h_ref, oracle.row_scales(len(rows), g=gh))
+    y2_chain_ref = oracle.gemm(hc_ref, hsf_ref, gh, wdc, wdsf, gcol_d)
+    got = oracle.bf16_bits_to_f64(gu.host_bits(y2[rows_t].contiguous()))
+    assert np.linalg.norm(got - y2_chain_ref) / np.linalg.norm(y2_chain_ref) <= 3e-3
+    assert (hc_ref == hc).mean() > 0.999

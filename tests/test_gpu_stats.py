@@ -1,5 +1,10 @@
-"""GPU parity for the NVFP4-granularity statistics: counts and the maximum exact, the three sums
-equal to the oracle's up to the order in which block results are added (double precision)."""
+"""GPU parity for the NVFP4-granularity statistics against the oracle's float64 definition.  The
+block count and the maximum are exact.  The kernel forms each block's sums in binary32 (16 fused
+multiply-adds: relative error below 16 * 2^-24 ~ 1e-6 per block, less in the total) and its
+dequantized value through one extra binary32 rounding of e4m3 * g (2^-24 relative on x_hat, i.e.
+about 1e-6 on an error that is a tenth of x): tolerances 5e-6 on sum x^2 and sum x^4, 2e-5 on
+sum err^2.  The 1-hot count compares bmax^2 * 16 with 9 * (binary32 block sum): a block within
+1e-6 of the threshold may fall on the other side, so the count may differ by a few in a million."""
 import numpy as np
 import pytest
 import torch
@@ -17,9 +22,10 @@ def _case(x_bits, g=None):
         _, g = oracle.calibrate(x_bits)
     want = oracle.stats_raw(x_bits, g)
     got = nv.nvfp4_tensor_stats(gu.dev_bf16(x_bits), gu.dev_f32(g)).cpu().numpy()
-    assert got[3] == want[3] and got[4] == want[4] and got[5] == want[5], (got, want)
-    for i in range(3):
-        assert abs(got[i] - want[i]) <= 1e-11 * abs(want[i]) + 1e-300, (i, got[i], want[i])
+    assert got[3] == want[3] and got[4] == want[4], (got, want)
+    assert abs(got[5] - want[5]) <= 1 + 5e-6 * want[4], (got, want)
+    for i, tol in ((0, 5e-6), (1, 5e-6), (2, 2e-5)):
+        assert abs(got[i] - want[i]) <= tol * abs(want[i]) + 1e-300, (i, got[i], want[i])
     return oracle.derive_stats(got[:6], x_bits.size)
 
 

@@ -113,7 +113,7 @@ def test_round_trip_error_bound():
 
 
 def test_outlier_only_touches_its_own_block():
-    # "an outlier degrades only its own 15 neighbors"
+    # the paper's locality remark: an outlier can only hurt the other fifteen values of its block
     rng = np.random.default_rng(4)
     x = _rand_bits(rng, 8, 128, spread=0.5)
     g = np.float32(0.01)

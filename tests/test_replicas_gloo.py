@@ -57,3 +57,18 @@ def test_single_rank_needs_no_process_group(monkeypatch):
     assert r.world == 1 and r.max_over_ranks(7.5) == 7.5 and r.aggregate(2.0, 1000.0) == 2.0
     r.barrier()
     r.close()
+
+
+def test_spawn_replicas_starts_one_process_per_rank(tmp_path):
+    # what `bench.py --gpus N` does when nobody exported RANK / WORLD_SIZE: N children, rank 0's line is the output
+    sys.path.insert(0, ROOT)
+    from paper_2609_04098_b200.replicas import spawn_replicas
+    script = tmp_path / "worker.py"
+    script.write_text(WORKER + "\nopen(os.environ['OUT_DIR'] + '/rank%d' % r.rank, 'w').write(str(r.world))\n")
+    for k in ("RANK", "LOCAL_RANK", "WORLD_SIZE"):
+        os.environ.pop(k, None)
+    rc = spawn_replicas(2, [sys.executable, str(script)], extra_env={"REPO_ROOT": ROOT, "OUT_DIR": str(tmp_path)},
+                        timeout=120)
+    assert rc == 0
+    assert (tmp_path / "rank0").read_text() == "2" and (tmp_path / "rank1").read_text() == "2"
+    assert spawn_replicas(2, [sys.executable, "-c", "import os, sys; sys.exit(3 if os.environ['RANK'] == '1' else 0)"]) == 3
