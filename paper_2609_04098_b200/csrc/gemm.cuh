@@ -21,11 +21,10 @@
 //   warp 5      TMA producer for W, same;
 //   warp 6      one thread (leader CTA only, in a pair) issues, per K=64 step, the three
 //               tcgen05.cp that bring that step's scale atoms from shared memory to TMEM
-//               and then the tcgen05.mma kind::mxf4nvf4.  Measured on B200: an MMA of
-//               N=256 takes 128 cycles, a tcgen05.cp 64 cycles, and the copies run beside
-//               the MMAs, so the pipe settles at ~196 cycles per step.  (Moving the scales
-//               with ld.shared + tcgen05.st from other warps was tried: the loads starve
-//               behind the tensor core's own shared-memory reads.)
+//               and then the tcgen05.mma kind::mxf4nvf4.  Measured on B200 (one SM, operands in
+//               shared memory): an MMA of N=256 occupies the tensor pipe for 128 cycles and the
+//               three copies add ~4 cycles when the issuing thread keeps up; what decides
+//               whether it keeps up is the SHAPE of the issuing code (see the loop).
 // Every mbarrier wait is bounded (ptx.cuh); a CTA that gives up raises a status word and
 // tells its partner instead of hanging.
 #pragma once
@@ -237,16 +236,18 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
     } else if (warp == 6) {
         // ------------------------------------------------------------ MMA issuer
-        // The tensor pipe accepts only about one instruction ahead of the one it is executing, so
-        // the instruction stream between two MMAs has to be short: the ring of stages is unrolled
-        // (every shared-memory and TMEM address is base + compile-time constant), descriptors are
-        // a fixed high word and an incremented low word, there are no divisions, and the next
-        // stage's barrier is polled before the current stage's last MMA.  The whole warp walks
-        // the loop so that all of this stays warp-uniform (tcgen05 operands are uniform
-        // registers; computed under a single-lane branch they cost a vector->uniform move chain
-        // per issue); one elected lane, the same throughout, issues.
+        // Issue-side rules (all measured on B200): the thread that issues tcgen05 work has to stay in
+        // warp-convergent code -- inside a single-lane branch every operand pays a vector-to-uniform
+        // move and [3 copies + 1 MMA] cost ~200 cycles to issue, in convergent code with only the
+        // instruction predicated they cost ~135 and the tensor pipe (128 cycles per MMA) stays busy.
+        // So the whole warp walks the loop; `lp` is non-zero in one elected lane, the same throughout.
+        // The ring of stages is unrolled (every shared-memory and TMEM address is base + compile-time
+        // constant; a rolled loop with run-time stage addresses measured 8 % slower), descriptors are a
+        // fixed high word and an incremented low word, there are no divisions, and the next stage's
+        // barrier is polled right after the first MMA of the current stage has been queued, when the
+        // pipe has most work ahead of it.
         if (rank == 0) {
-            const bool leader = ptx::elect_one();
+            const uint32_t lp = ptx::elect_one() ? 1u : 0u;
             // E2M1 x E2M1, E4M3 scales, K-major A and B; M = 128 (single) or 256 (pair), N = BN
             constexpr uint32_t idesc = (1u << 7) | (1u << 10) | (static_cast<uint32_t>(BN >> 3) << 17) |
                                        (static_cast<uint32_t>((PAIR ? 256 : 128) >> 4) << 24);
@@ -272,8 +273,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                         const uint32_t dep = C::OVERLAP ? tl - 1u : tl - 2u;
                         if (tl >= (C::OVERLAP ? 1u : 2u)) {
                             if (!ptx::mbar_wait_bounded(&tempty[dep & 1u], (dep >> 1) & 1u, abort_flag, p.wait_limit_ns, peer_abort)) { ok = false; break; }
+                            ptx::tc_fence_after();
                         }
-                        if (have_full) ptx::tc_fence_after();
                     }
                     if (!have_full) {
                         if (!ptx::mbar_wait_bounded(&full[s], ph, abort_flag, p.wait_limit_ns, peer_abort)) { ok = false; break; }
@@ -289,48 +290,42 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
                     for (int j = 0; j < kStepsPerStage; ++j) {
                         if (j < steps) {
-                            if (j == kStepsPerStage - 1 && it + 1 < total_it) {
-                                // while the earlier steps run: has the next stage landed?
-                                const int ns = (s + 1 == STAGES) ? 0 : s + 1;
-                                if (ptx::mbar_try_wait(&full[ns], ns == 0 ? ph ^ 1u : ph)) { ptx::tc_fence_after(); have_full = true; }
-                            }
                             // this step's scale atoms: shared -> TMEM (32 rows x 16 bytes each, replicated into
                             // the four lane quarters), then the MMA that reads them
-                            if (leader) {
-                                const uint32_t sf_enc = st_enc + ((C::A_BYTES + C::B_BYTES + j * 512) >> 4);
-                                if (PAIR) {
-                                    ptx::tc_cp_32x128b_warpx4_pair(sfa_t + j * 4, desc(sf_enc, kScaleHi));
-                                    ptx::tc_cp_32x128b_warpx4_pair(sfb_t + j * (BN / 32), desc(sf_enc + (C::SFA_BYTES >> 4), kScaleHi));
-                                    if (C::NB_BANDS == 2)
-                                        ptx::tc_cp_32x128b_warpx4_pair(sfb_t + j * (BN / 32) + 4,
-                                                                       desc(sf_enc + ((C::SFA_BYTES + kStepsPerStage * 512) >> 4), kScaleHi));
-                                } else {
-                                    ptx::tc_cp_32x128b_warpx4(sfa_t + j * 4, desc(sf_enc, kScaleHi));
-                                    ptx::tc_cp_32x128b_warpx4(sfb_t + j * (BN / 32), desc(sf_enc + (C::SFA_BYTES >> 4), kScaleHi));
-                                    if (C::NB_BANDS == 2)
-                                        ptx::tc_cp_32x128b_warpx4(sfb_t + j * (BN / 32) + 4,
-                                                                  desc(sf_enc + ((C::SFA_BYTES + kStepsPerStage * 512) >> 4), kScaleHi));
-                                }
+                            const uint32_t sf_enc = st_enc + ((C::A_BYTES + C::B_BYTES + j * 512) >> 4);
+                            // advancing K by 64 elements = 32 bytes inside the 128-byte swizzle row
+                            const uint64_t a_desc = desc((st_enc + j * 2) | kCodeLoFlags, kCodeHi);
+                            const uint64_t b_desc = desc((st_enc + (C::A_BYTES >> 4) + j * 2) | kCodeLoFlags, kCodeHi);
+                            const uint32_t accum = (j == 0) ? (kt != 0u ? 1u : 0u) : 1u;
+                            if (PAIR) {
+                                ptx::tc_cp_32x128b_warpx4_pair_if(sfa_t + j * 4, desc(sf_enc, kScaleHi), lp);
+                                ptx::tc_cp_32x128b_warpx4_pair_if(sfb_t + j * (BN / 32), desc(sf_enc + (C::SFA_BYTES >> 4), kScaleHi), lp);
+                                if (C::NB_BANDS == 2)
+                                    ptx::tc_cp_32x128b_warpx4_pair_if(sfb_t + j * (BN / 32) + 4,
+                                                                      desc(sf_enc + ((C::SFA_BYTES + kStepsPerStage * 512) >> 4), kScaleHi), lp);
+                                ptx::tc_mma_nvf4_pair_if(d_tmem, a_desc, b_desc, idesc, sfa_t + j * 4, sfb_t + j * (BN / 32), accum, lp);
+                            } else {
+                                ptx::tc_cp_32x128b_warpx4_if(sfa_t + j * 4, desc(sf_enc, kScaleHi), lp);
+                                ptx::tc_cp_32x128b_warpx4_if(sfb_t + j * (BN / 32), desc(sf_enc + (C::SFA_BYTES >> 4), kScaleHi), lp);
+                                if (C::NB_BANDS == 2)
+                                    ptx::tc_cp_32x128b_warpx4_if(sfb_t + j * (BN / 32) + 4,
+                                                                 desc(sf_enc + ((C::SFA_BYTES + kStepsPerStage * 512) >> 4), kScaleHi), lp);
+                                ptx::tc_mma_nvf4_if(d_tmem, a_desc, b_desc, idesc, sfa_t + j * 4, sfb_t + j * (BN / 32), accum, lp);
                             }
-                            if (leader) {
-                                // advancing K by 64 elements = 32 bytes inside the 128-byte swizzle row
-                                const uint64_t a_desc = desc((st_enc + j * 2) | kCodeLoFlags, kCodeHi);
-                                const uint64_t b_desc = desc((st_enc + (C::A_BYTES >> 4) + j * 2) | kCodeLoFlags, kCodeHi);
-                                const uint32_t accum = (j == 0) ? (kt != 0u ? 1u : 0u) : 1u;
-                                if (PAIR) ptx::tc_mma_nvf4_pair(d_tmem, a_desc, b_desc, idesc, sfa_t + j * 4, sfb_t + j * (BN / 32), accum);
-                                else      ptx::tc_mma_nvf4(d_tmem, a_desc, b_desc, idesc, sfa_t + j * 4, sfb_t + j * (BN / 32), accum);
+                            if (j == 0 && it + 1 < total_it) {
+                                // with this stage's first MMA queued: has the next stage landed?
+                                const int ns = (s + 1 == STAGES) ? 0 : s + 1;
+                                if (ptx::mbar_try_wait(&full[ns], ns == 0 ? ph ^ 1u : ph)) { ptx::tc_fence_after(); have_full = true; }
                             }
                         }
                     }
                     // stage reusable once these MMAs have read it; after the last K tile the accumulator is complete
-                    if (leader) {
-                        if (PAIR) {
-                            ptx::tc_commit_pair(&empty[s], 3);
-                            if (last_kt) ptx::tc_commit_pair(&tfull[acc], 3);
-                        } else {
-                            ptx::tc_commit(&empty[s]);
-                            if (last_kt) ptx::tc_commit(&tfull[acc]);
-                        }
+                    if (PAIR) {
+                        ptx::tc_commit_pair_if(&empty[s], 3, lp);
+                        if (last_kt) ptx::tc_commit_pair_if(&tfull[acc], 3, lp);
+                    } else {
+                        ptx::tc_commit_if(&empty[s], lp);
+                        if (last_kt) ptx::tc_commit_if(&tfull[acc], lp);
                     }
                     ++it;
                     if (last_kt) { kt = 0; ++tl; } else { ++kt; }
@@ -339,7 +334,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             }
             if (!ok) {
                 // let issued MMAs finish before TMEM is freed
-                if (leader) { if (PAIR) ptx::tc_commit_pair(drain, 1); else ptx::tc_commit(drain); }
+                if (PAIR) ptx::tc_commit_pair_if(drain, 1, lp); else ptx::tc_commit_if(drain, lp);
                 for (int spin = 0; spin < (1 << 16) && !ptx::mbar_try_wait(drain, 0u); ++spin) {}
             }
         }

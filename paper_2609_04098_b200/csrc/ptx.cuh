@@ -61,6 +61,23 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 
+// One poll by the lanes whose `pred` is non-zero (the others do not touch the barrier and get false).
+__device__ __forceinline__ bool mbar_try_wait_if(uint64_t* bar, uint32_t parity, uint32_t pred) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred q, P;\n\t"
+        "setp.ne.b32 q, %3, 0;\n\t"
+        "mov.pred P, 0;\n\t"
+        "@q mbarrier.try_wait.parity.shared::cta.b64 P, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, P;\n\t"
+        "}\n"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(pred)
+        : "memory");
+    return ok != 0;
+}
+
 // Bounded wait: spins on try_wait; every 32 failed polls it looks at the CTA's
 // abort flag and at the wall clock.  Returns false (and raises the abort flag) if
 // `limit_ns` passes or another role already gave up, so no wait can hang the GPU.
@@ -265,6 +282,54 @@ __device__ __forceinline__ void tc_mma_nvf4_pair(uint32_t d_tmem, uint64_t a_des
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
         : "memory");
 }
+// ---- predicated forms.  The thread that issues tcgen05 work must stay in warp-convergent code:
+// measured on B200, the same instruction sequence costs the issuing thread ~200 cycles per
+// [3 copies + 1 MMA] when it sits inside a single-lane branch and ~135 cycles when the whole warp
+// walks the code and only the instruction itself is predicated on `pred` (non-zero in exactly one
+// lane).  Every operand is then computed by all lanes alike.
+__device__ __forceinline__ void tc_cp_32x128b_warpx4_if(uint32_t taddr, uint64_t smem_desc, uint32_t pred) {
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %2, 0;\n\t"
+                 "@q tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;\n\t}\n" ::"r"(taddr), "l"(smem_desc), "r"(pred) : "memory");
+}
+__device__ __forceinline__ void tc_cp_32x128b_warpx4_pair_if(uint32_t taddr, uint64_t smem_desc, uint32_t pred) {
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %2, 0;\n\t"
+                 "@q tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;\n\t}\n" ::"r"(taddr), "l"(smem_desc), "r"(pred) : "memory");
+}
+__device__ __forceinline__ void tc_mma_nvf4_if(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                               uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate, uint32_t pred) {
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p, q;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "setp.ne.b32 q, %7, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::mxf4nvf4.block_scale.scale_vec::4X [%0], %1, %2, %3, [%5], [%6], p;\n\t"
+        "}\n"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem), "r"(pred)
+        : "memory");
+}
+__device__ __forceinline__ void tc_mma_nvf4_pair_if(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                                    uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate, uint32_t pred) {
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p, q;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "setp.ne.b32 q, %7, 0;\n\t"
+        "@q tcgen05.mma.cta_group::2.kind::mxf4nvf4.block_scale.scale_vec::4X [%0], %1, %2, %3, [%5], [%6], p;\n\t"
+        "}\n"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem), "r"(pred)
+        : "memory");
+}
+__device__ __forceinline__ void tc_commit_if(uint64_t* bar, uint32_t pred) {
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %1, 0;\n\t"
+                 "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}\n"
+                 ::"r"(smem_u32(bar)), "r"(pred) : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair_if(uint64_t* bar, uint16_t cta_mask, uint32_t pred) {
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %2, 0;\n\t"
+                 "@q tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;\n\t}\n"
+                 ::"r"(smem_u32(bar)), "h"(cta_mask), "r"(pred) : "memory");
+}
+
 // 32 lanes x 32 consecutive 32-bit columns -> 32 registers per thread (thread i = lane i
 // of this warp's TMEM quarter).
 __device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32]) {
