@@ -191,7 +191,7 @@ struct GemmMaps {
     CUtensorMap a, b, sfa, sfb, y;
 };
 
-template <int BN, int STAGES, bool PAIR>
+template <int BN, int STAGES, bool PAIR, bool FULLK>
 nvfp4_status launch_gemm(const GemmMaps& tm, GemmParams& p, int sm_count, cudaStream_t stream) {
     using C = GemmCfg<BN, STAGES, PAIR>;
     static std::mutex mu;
@@ -231,14 +231,14 @@ nvfp4_status launch_gemm(const GemmMaps& tm, GemmParams& p, int sm_count, cudaSt
         std::lock_guard<std::mutex> lock(mu);
         units = max_units[dev];
         if (units == 0) {
-            if (cudaFuncSetAttribute(gemm_kernel<BN, STAGES, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            if (cudaFuncSetAttribute(gemm_kernel<BN, STAGES, PAIR, FULLK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      C::SMEM_BYTES) != cudaSuccess)
                 return NVFP4_ERR_CUDA;
             units = PAIR ? sm_count / 2 : sm_count;
             if (PAIR) {
                 cfg.gridDim = dim3(static_cast<unsigned>(sm_count & ~1), 1, 1);
                 int n = 0;
-                if (cudaOccupancyMaxActiveClusters(&n, gemm_kernel<BN, STAGES, PAIR>, &cfg) == cudaSuccess && n >= 1) {
+                if (cudaOccupancyMaxActiveClusters(&n, gemm_kernel<BN, STAGES, PAIR, FULLK>, &cfg) == cudaSuccess && n >= 1) {
                     if (n < units) units = n;
                 } else {
                     cudaGetLastError();
@@ -249,7 +249,7 @@ nvfp4_status launch_gemm(const GemmMaps& tm, GemmParams& p, int sm_count, cudaSt
     }
     const int64_t use = tiles < units ? tiles : units;
     cfg.gridDim = dim3(static_cast<unsigned>((PAIR ? 2 : 1) * use), 1, 1);
-    cudaError_t e = cudaLaunchKernelEx(&cfg, gemm_kernel<BN, STAGES, PAIR>, tm.a, tm.b, tm.sfa, tm.sfb, tm.y, p);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, gemm_kernel<BN, STAGES, PAIR, FULLK>, tm.a, tm.b, tm.sfa, tm.sfb, tm.y, p);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return e == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
@@ -673,10 +673,11 @@ nvfp4_status linear_impl(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const 
         p.wait_limit_ns = lim != 0 ? lim : kWaitLimitNs;
     }
     cudaStream_t s = as_stream(stream);
+    const bool fullk = (K % 256) == 0;
     switch (bn) {
-        case 128: return launch_gemm<128, 5, false>(tm, p, info.sm_count, s);
-        case 256: return launch_gemm<256, 3, false>(tm, p, info.sm_count, s);
-        case 2: return launch_gemm<256, 5, true>(tm, p, info.sm_count, s);
+        case 128: return fullk ? launch_gemm<128, 5, false, true>(tm, p, info.sm_count, s) : launch_gemm<128, 5, false, false>(tm, p, info.sm_count, s);
+        case 256: return fullk ? launch_gemm<256, 3, false, true>(tm, p, info.sm_count, s) : launch_gemm<256, 3, false, false>(tm, p, info.sm_count, s);
+        case 2: return fullk ? launch_gemm<256, 5, true, true>(tm, p, info.sm_count, s) : launch_gemm<256, 5, true, false>(tm, p, info.sm_count, s);
         default: return NVFP4_ERR_SHAPE;
     }
 }
