@@ -130,8 +130,9 @@ nvfp4_status nvfp4_quantize_act(const void* d_x, int64_t M, int64_t K, int64_t l
  * The paper fixes no arithmetic for the activation (it is upstream of the quantized linears, in
  * bf16).  The kernel evaluates it in binary32 with the hardware's approximate exp2 and
  * reciprocal; the bf16 result equals the correctly rounded definition for all but a small
- * fraction of elements and is never more than one bf16 ulp away.  Codes and scales are the exact
- * quantization of the h the kernel formed.
+ * fraction of elements and is never more than one bf16 ulp away (results below about 2^-100 in
+ * magnitude, from gates below -88, come out as zeros of the right sign).  Codes and scales are the
+ * exact quantization of the h the kernel formed.
  *   d_gate_up  bf16 [M, 2*inner], gate in columns [0, inner), up in [inner, 2*inner); row
  *              stride ld >= 2*inner; 32-byte aligned, ld % 16 == 0, inner % 16 == 0
  *   d_g        in: global scale of h (calibrated offline, as for any activation)
@@ -178,6 +179,47 @@ nvfp4_status nvfp4_quantize_weight(const void* d_w, int64_t N, int64_t K, int64_
                                    const nvfp4_segment* segs, int nseg, float* d_g_seg,
                                    int calibrate_segments, uint8_t* d_codes, uint8_t* d_sf,
                                    nvfp4_sf_layout layout, void* stream);
+
+/*
+ * Weight quantization for the MLP's fused gate/up projection with the output rows INTERLEAVED
+ * 16 by 16: output rows 32 b .. 32 b + 15 are gate rows 16 b .. 16 b + 15 and rows 32 b + 16 ..
+ * 32 b + 31 the matching up rows.  Each module keeps its own global scale (paper: Section 6, one
+ * FP32 global scale per linear module).  Quantization is per row, so codes and scale bytes are
+ * those nvfp4_quantize_weight gives for the same rows; only the row order differs.  A GEMM
+ * against weights in this order (nvfp4_linear_swiglu) produces, per 32 output columns, the 16
+ * gate and 16 up values of one 16-element block of silu(gate) * up.
+ *   d_w           bf16 [2 * inner, K]: gate rows [0, inner), then up rows [inner, 2 * inner); row stride ld
+ *   d_g_gate_up   device float[2]: INPUT when calibrate_segments == 0, else OUTPUT (amax / 2688 of each module)
+ *   d_codes       out [2 * inner, K / 2];  d_sf out nvfp4_sf_bytes(2 * inner, K, NVFP4_SF_MMA)
+ * Errors: as nvfp4_quantize_weight; inner % 16 != 0 is NVFP4_ERR_SHAPE.
+ */
+nvfp4_status nvfp4_quantize_weight_gate_up(const void* d_w, int64_t inner, int64_t K, int64_t ld,
+                                           float* d_g_gate_up, int calibrate_segments,
+                                           uint8_t* d_codes, uint8_t* d_sf, void* stream);
+
+/*
+ * The MLP's gate/up projection with SwiGLU and the activation quantization of the down
+ * projection's input inside the GEMM epilogue (paper: Background -- the MLP is among the 496
+ * quantized linears; Section 9 names activation quantization as the overhead to remove): the
+ * gate/up output is never written in bf16, only the NVFP4 codes and scale bytes of
+ *     h = bf16_rne( silu(gate) * up ),  gate = bf16_rne(acc * g_a * g_gate),  up = bf16_rne(acc * g_a * g_up)
+ * exactly as nvfp4_linear followed by nvfp4_swiglu_quantize would produce them (same roundings).
+ *   d_a_codes/d_a_sf   activations [M, K] (NVFP4_SF_MMA);  d_g_a their global scale
+ *   d_w_codes/d_w_sf   from nvfp4_quantize_weight_gate_up;  d_g_gate_up device float[2]
+ *   d_g_h              in: global scale of h (calibrated offline, as for any activation)
+ *   d_h_codes          out [M, inner / 2], 16-byte aligned
+ *   d_h_sf             out nvfp4_sf_bytes(M, inner, NVFP4_SF_MMA) bytes (every byte is written)
+ *   d_dbg_y, d_dbg_h   optional (may be NULL), testing aids, 32-byte aligned: bf16 [M, 2 * inner] gate/up in the
+ *                      interleaved column order, and bf16 [M, inner] the tensor h that was quantized
+ *   d_workspace        as for nvfp4_linear (256 bytes suffice)
+ * Requirements: K % 64 == 0, inner % 64 == 0.  Errors and the status word as for nvfp4_linear.
+ */
+nvfp4_status nvfp4_linear_swiglu(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const float* d_g_a,
+                                 int64_t M, int64_t K,
+                                 const uint8_t* d_w_codes, const uint8_t* d_w_sf, int64_t inner,
+                                 const float* d_g_gate_up, const float* d_g_h,
+                                 uint8_t* d_h_codes, uint8_t* d_h_sf, void* d_dbg_y, void* d_dbg_h,
+                                 void* d_workspace, size_t workspace_bytes, void* stream);
 
 /*
  * Checkpoint-side repair (paper: Section 6, the fix applied to the released checkpoint: every

@@ -25,7 +25,7 @@ MAX_SEGMENTS = 32
 
 EXPORTS = (
     "nvfp4_sf_bytes", "nvfp4_calibrate", "nvfp4_quantize_act", "nvfp4_swiglu_quantize", "nvfp4_rmsnorm_quantize",
-    "nvfp4_quantize_weight",
+    "nvfp4_quantize_weight", "nvfp4_quantize_weight_gate_up", "nvfp4_linear_swiglu",
     "nvfp4_harmonize_scales", "nvfp4_tensor_stats", "nvfp4_linear", "nvfp4_linear_workspace_bytes", "nvfp4_linear_bf16",
     "nvfp4_linear_bf16_workspace_bytes", "nvfp4_linear_bf16_static", "nvfp4_static_status", "nvfp4_workspace_reset", "nvfp4_device_status",
     "nvfp4_set_wait_limit_ns", "nvfp4_selftest_bounded_wait", "nvfp4_launch_count", "nvfp4_set_gemm_variant", "nvfp4_gemm_variants", "nvfp4_status_string",
@@ -67,6 +67,10 @@ def lib() -> ctypes.CDLL:
     L.nvfp4_rmsnorm_quantize.argtypes = [vp, i64, i64, i64, vp, ctypes.c_float, vp, vp, vp, i32, vp, vp]
     L.nvfp4_quantize_weight.restype = i32
     L.nvfp4_quantize_weight.argtypes = [vp, i64, i64, i64, segp, i32, vp, i32, vp, vp, i32, vp]
+    L.nvfp4_quantize_weight_gate_up.restype = i32
+    L.nvfp4_quantize_weight_gate_up.argtypes = [vp, i64, i64, i64, vp, i32, vp, vp, vp]
+    L.nvfp4_linear_swiglu.restype = i32
+    L.nvfp4_linear_swiglu.argtypes = [vp, vp, vp, i64, i64, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     L.nvfp4_harmonize_scales.restype = i32
     L.nvfp4_harmonize_scales.argtypes = [vp, i64, i64, i32, segp, vp, i32, vp, vp, vp]
     L.nvfp4_tensor_stats.restype = i32
@@ -228,6 +232,35 @@ def nvfp4_quantize_weight(w: torch.Tensor, segments, g_seg: Optional[torch.Tenso
                                        calibrate, _ptr(codes), _ptr(sf), layout, _stream(stream)),
            "nvfp4_quantize_weight")
     return codes, sf, g_seg
+
+
+def nvfp4_quantize_weight_gate_up(w: torch.Tensor, g_gate_up: Optional[torch.Tensor] = None, out=None, stream=None):
+    """bf16 [2I, K] (gate rows, then up rows) -> (codes, scale bytes, g[2]) with the rows interleaved 16 by 16,
+    the order ``nvfp4_linear_swiglu`` expects.  ``g_gate_up=None`` calibrates each module on the device."""
+    assert w.is_cuda and w.dtype == torch.bfloat16 and w.dim() == 2 and w.stride(1) == 1 and w.shape[0] % 2 == 0
+    N, K = w.shape
+    calibrate = 0
+    if g_gate_up is None:
+        g_gate_up = torch.empty(2, dtype=torch.float32, device=w.device)
+        calibrate = 1
+    codes, sf = out if out is not None else alloc_quantized(N, K, w.device, SF_MMA)
+    _check(lib().nvfp4_quantize_weight_gate_up(_ptr(w), N // 2, K, w.stride(0), _ptr(g_gate_up), calibrate, _ptr(codes),
+                                               _ptr(sf), _stream(stream)), "nvfp4_quantize_weight_gate_up")
+    return codes, sf, g_gate_up
+
+
+def nvfp4_linear_swiglu(a_codes, a_sf, g_a, w_codes, w_sf, g_gate_up, g_h, workspace, out=None, stream=None,
+                        dbg_y: Optional[torch.Tensor] = None, dbg_h: Optional[torch.Tensor] = None):
+    """Gate/up GEMM with SwiGLU and the quantization of h = silu(gate) * up in its epilogue: returns
+    (codes u8 [M, I/2], scale bytes) of h, ready for the down projection.  ``dbg_y`` (bf16 [M, 2I], interleaved
+    columns) and ``dbg_h`` (bf16 [M, I]) are optional testing outputs."""
+    M, K = a_codes.shape[0], a_codes.shape[1] * 2
+    inner = w_codes.shape[0] // 2
+    codes, sf = out if out is not None else alloc_quantized(M, inner, a_codes.device, SF_MMA)
+    _check(lib().nvfp4_linear_swiglu(_ptr(a_codes), _ptr(a_sf), _ptr(g_a), M, K, _ptr(w_codes), _ptr(w_sf), inner,
+                                     _ptr(g_gate_up), _ptr(g_h), _ptr(codes), _ptr(sf), _ptr(dbg_y), _ptr(dbg_h),
+                                     _ptr(workspace), workspace.numel(), _stream(stream)), "nvfp4_linear_swiglu")
+    return codes, sf
 
 
 def nvfp4_harmonize_scales(w_sf: torch.Tensor, N: int, K: int, segments, g_seg: torch.Tensor,

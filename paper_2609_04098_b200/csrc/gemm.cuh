@@ -36,6 +36,7 @@
 
 #include "../../include/nvfp4.h"
 #include "ptx.cuh"
+#include "quantize.cuh"
 
 namespace nvfp4 {
 
@@ -63,7 +64,17 @@ struct GemmParams {
     int32_t nseg;
     int32_t seg_end[NVFP4_MAX_SEGMENTS];
     uint64_t wait_limit_ns;
+    // fused SwiGLU + quantize epilogue (EPI == kEpiSwiglu): the W rows are gate/up interleaved 16 by 16,
+    // N = 2 * inner; the epilogue writes NVFP4 codes and scales of h = silu(gate) * up instead of Y
+    const float* g_h;        // device scalar: global scale of h
+    uint8_t* h_codes;        // [M, inner / 2]
+    uint8_t* h_sf;           // tensor-core scale layout of an [M, inner] tensor
+    int32_t h_katoms;        // inner / 64
+    int32_t inner;
+    void* dbg_y;             // optional testing outputs: bf16 [M, 2 * inner] (interleaved columns) ...
+    void* dbg_h;             // ... and bf16 [M, inner]
 };
+constexpr int kEpiPlain = 0, kEpiSwiglu = 1;
 
 constexpr int kGemmThreads = 224;
 constexpr int kBM = 128;
@@ -115,7 +126,10 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 
 // FULLK: K is a multiple of 256, so every stage holds four K-steps and the issue loop has no
 // per-step condition (a run-time branch around each step costs the loop ~20 %, measured).
-template <int BN, int STAGES, bool PAIR, bool FULLK>
+// EPI: kEpiPlain writes Y; kEpiSwiglu (BN = 256 only) turns every 32 accumulator columns -- 16 gate
+// and 16 up values of one row -- into one 16-element block of h = bf16(silu(bf16(gate)) * bf16(up))
+// and writes its NVFP4 codes and scale byte: the 4 bytes per element that Y would cost become 0.5625.
+template <int BN, int STAGES, bool PAIR, bool FULLK, int EPI = kEpiPlain>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const __grid_constant__ CUtensorMap tmSFA, const __grid_constant__ CUtensorMap tmSFB,
@@ -387,6 +401,73 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * C::ACC_STRIDE;
             const int32_t row0 = (PAIR ? 2 * um + static_cast<int32_t>(rank) : um) * kBM + quarter * 32;
             constexpr int NP = BN / kOutPieceCols;
+            if (EPI == kEpiSwiglu) {
+                // ---- fused SwiGLU + quantize.  Piece order as in the plain epilogue (the columns shared by
+                // the two accumulators go first); each piece of 64 columns holds two blocks of h.
+                const float a_gate = __fmul_rn(g_a, __ldg(p.g_seg)), a_up = __fmul_rn(g_a, __ldg(p.g_seg + 1));
+                const float g_h = __ldg(p.g_h);
+                const float c1_h = __fdiv_rn(1.0f, __fmul_rn(6.0f, g_h));
+                const int32_t row = row0 + lane;
+                const int32_t m_pad = (p.M + 127) & ~127;
+                const int first_piece = (C::OVERLAP && acc == 0u) ? NP - 1 : 0;
+                uint32_t ra[64], rb[64];
+                ptx::tmem_ld_32x64(t_row + first_piece * kOutPieceCols, ra);
+#pragma unroll
+                for (int k = 0; k < NP; ++k) {
+                    uint32_t (&cur)[64] = (k & 1) ? rb : ra;
+                    uint32_t (&nxt)[64] = (k & 1) ? ra : rb;
+                    const int pc = (first_piece + k) % NP;
+                    ptx::tmem_ld_wait();
+                    if (k + 1 < NP) ptx::tmem_ld_32x64(t_row + ((pc + 1) % NP) * kOutPieceCols, nxt);
+                    if (C::OVERLAP ? (k == 0) : (k + 1 == NP)) {
+                        ptx::tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) {
+                            if (PAIR) ptx::mbar_arrive_cluster(leader_tempty + acc * 8u);
+                            else      ptx::mbar_arrive(&tempty[acc]);
+                        }
+                    }
+                    const int32_t col0 = n0 + pc * kOutPieceCols;             // interleaved column of this piece
+                    if (col0 < p.N && row < m_pad) {
+                    const int32_t hc0 = col0 >> 1;                            // first h column of this piece (32 of them)
+                    uint2 words[2];
+                    uint32_t s8[2];
+#pragma unroll
+                    for (int b = 0; b < 2; ++b) {
+                        uint32_t hw[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            // gate / up rounded to bf16 exactly as the plain epilogue would store them
+                            const float g0 = __bfloat162float(__float2bfloat16_rn(__fmul_rn(__uint_as_float(cur[b * 32 + 2 * i]), a_gate)));
+                            const float g1 = __bfloat162float(__float2bfloat16_rn(__fmul_rn(__uint_as_float(cur[b * 32 + 2 * i + 1]), a_gate)));
+                            const float u0 = __bfloat162float(__float2bfloat16_rn(__fmul_rn(__uint_as_float(cur[b * 32 + 16 + 2 * i]), a_up)));
+                            const float u1 = __bfloat162float(__float2bfloat16_rn(__fmul_rn(__uint_as_float(cur[b * 32 + 16 + 2 * i + 1]), a_up)));
+                            hw[i] = pack_bf16x2(silu_mul(g0, u0), silu_mul(g1, u1));
+                        }
+                        words[b] = quantize_block(hw, g_h, c1_h, s8[b]);
+                        if (p.dbg_h != nullptr && row < p.M)
+                            stg256(reinterpret_cast<uint16_t*>(p.dbg_h) + static_cast<int64_t>(row) * p.inner + hc0 + b * 16, hw);
+                    }
+                    const int32_t kb0 = hc0 >> 4;                             // even: both scale bytes sit in one 16-bit word
+                    uint8_t* sfp = p.h_sf + (static_cast<int64_t>(row >> 7) * p.h_katoms + (kb0 >> 2)) * 512 + (row & 31) * 16 +
+                                   ((row & 127) >> 5) * 4 + (kb0 & 3);
+                    if (row < p.M) {
+                        *reinterpret_cast<uint4*>(p.h_codes + static_cast<int64_t>(row) * (p.inner >> 1) + (hc0 >> 1)) =
+                            make_uint4(words[0].x, words[0].y, words[1].x, words[1].y);
+                        *reinterpret_cast<uint16_t*>(sfp) = static_cast<uint16_t>(s8[0] | (s8[1] << 8));
+                        if (p.dbg_y != nullptr) {
+                            __nv_bfloat16* yr = reinterpret_cast<__nv_bfloat16*>(p.dbg_y) + static_cast<int64_t>(row) * p.N + col0;
+#pragma unroll
+                            for (int j = 0; j < 64; ++j)
+                                yr[j] = __float2bfloat16_rn(__fmul_rn(__uint_as_float(cur[j]), (j & 16) ? a_up : a_gate));
+                        }
+                    } else {
+                        *reinterpret_cast<uint16_t*>(sfp) = 0;                 // rows that pad the last 128-row band: zero scales
+                    }
+                    }
+                }
+                continue;
+            }
             if (split_k > 1u) {
                 // ---- split-K: add this item's partial sums to the tile's fp32 buffer; the last of
                 // the split_k arrivals (per lane quarter) finishes the tile

@@ -191,7 +191,7 @@ struct GemmMaps {
     CUtensorMap a, b, sfa, sfb, y;
 };
 
-template <int BN, int STAGES, bool PAIR, bool FULLK>
+template <int BN, int STAGES, bool PAIR, bool FULLK, int EPI = kEpiPlain>
 nvfp4_status launch_gemm(const GemmMaps& tm, GemmParams& p, int sm_count, cudaStream_t stream) {
     using C = GemmCfg<BN, STAGES, PAIR>;
     static std::mutex mu;
@@ -231,14 +231,14 @@ nvfp4_status launch_gemm(const GemmMaps& tm, GemmParams& p, int sm_count, cudaSt
         std::lock_guard<std::mutex> lock(mu);
         units = max_units[dev];
         if (units == 0) {
-            if (cudaFuncSetAttribute(gemm_kernel<BN, STAGES, PAIR, FULLK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            if (cudaFuncSetAttribute(gemm_kernel<BN, STAGES, PAIR, FULLK, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      C::SMEM_BYTES) != cudaSuccess)
                 return NVFP4_ERR_CUDA;
             units = PAIR ? sm_count / 2 : sm_count;
             if (PAIR) {
                 cfg.gridDim = dim3(static_cast<unsigned>(sm_count & ~1), 1, 1);
                 int n = 0;
-                if (cudaOccupancyMaxActiveClusters(&n, gemm_kernel<BN, STAGES, PAIR, FULLK>, &cfg) == cudaSuccess && n >= 1) {
+                if (cudaOccupancyMaxActiveClusters(&n, gemm_kernel<BN, STAGES, PAIR, FULLK, EPI>, &cfg) == cudaSuccess && n >= 1) {
                     if (n < units) units = n;
                 } else {
                     cudaGetLastError();
@@ -249,7 +249,7 @@ nvfp4_status launch_gemm(const GemmMaps& tm, GemmParams& p, int sm_count, cudaSt
     }
     const int64_t use = tiles < units ? tiles : units;
     cfg.gridDim = dim3(static_cast<unsigned>((PAIR ? 2 : 1) * use), 1, 1);
-    cudaError_t e = cudaLaunchKernelEx(&cfg, gemm_kernel<BN, STAGES, PAIR, FULLK>, tm.a, tm.b, tm.sfa, tm.sfb, tm.y, p);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, gemm_kernel<BN, STAGES, PAIR, FULLK, EPI>, tm.a, tm.b, tm.sfa, tm.sfb, tm.y, p);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return e == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
@@ -481,6 +481,31 @@ nvfp4_status nvfp4_quantize_weight(const void* d_w, int64_t N, int64_t K, int64_
     return quantize_impl(d_w, N, K, ld, d_g_seg, table, d_codes, d_sf, layout, info, as_stream(stream));
 }
 
+nvfp4_status nvfp4_quantize_weight_gate_up(const void* d_w, int64_t inner, int64_t K, int64_t ld, float* d_g_gate_up,
+                                           int calibrate_segments, uint8_t* d_codes, uint8_t* d_sf, void* stream) {
+    const int64_t N = 2 * inner;
+    nvfp4_status st = check_quantize_args(d_w, N, K, ld, d_g_gate_up, d_codes, d_sf, NVFP4_SF_MMA);
+    if (st != NVFP4_OK) return st;
+    if (inner <= 0 || (inner % 16) != 0 || N >= (1ll << 31)) return NVFP4_ERR_SHAPE;
+    DeviceInfo info;
+    st = check_arch(info);
+    if (st != NVFP4_OK) return st;
+    SegTable table;
+    std::memset(&table, 0, sizeof(table));
+    table.nseg = 2;
+    table.row_end[0] = static_cast<int32_t>(inner);
+    table.row_end[1] = static_cast<int32_t>(N);
+    table.il_inner = static_cast<int32_t>(inner);
+    if (calibrate_segments != 0) {
+        const uint16_t* w = reinterpret_cast<const uint16_t*>(d_w);
+        for (int i = 0; i < 2; ++i) {
+            st = nvfp4_calibrate(w + i * inner * ld, inner, K, ld, d_g_gate_up + i, nullptr, stream);
+            if (st != NVFP4_OK) return st;
+        }
+    }
+    return quantize_impl(d_w, N, K, ld, d_g_gate_up, table, d_codes, d_sf, NVFP4_SF_MMA, info, as_stream(stream));
+}
+
 nvfp4_status nvfp4_swiglu_quantize(const void* d_gate_up, int64_t M, int64_t inner, int64_t ld, const float* d_g,
                                    uint8_t* d_codes, uint8_t* d_sf, nvfp4_sf_layout layout, void* d_h, void* stream) {
     nvfp4_status st = check_quantize_args(d_gate_up, M, inner, ld, d_g, d_codes, d_sf, layout);
@@ -596,9 +621,9 @@ nvfp4_status linear_impl(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const 
                          int64_t K, const uint8_t* d_w_codes, const uint8_t* d_w_sf, int64_t N,
                          const nvfp4_segment* segs, const float* d_g_seg, int nseg, void* d_y, int64_t ldy,
                          uint32_t flags, void* d_workspace, size_t workspace_bytes, void* d_split, size_t split_bytes,
-                         void* stream, int64_t a_rows_alloc = 0) {
+                         void* stream, int64_t a_rows_alloc = 0, const GemmParams* fused = nullptr) {
     if (d_a_codes == nullptr || d_a_sf == nullptr || d_g_a == nullptr || d_w_codes == nullptr ||
-        d_w_sf == nullptr || d_g_seg == nullptr || d_y == nullptr)
+        d_w_sf == nullptr || d_g_seg == nullptr || (d_y == nullptr && fused == nullptr))
         return NVFP4_ERR_NULL;
     if (M < 0 || N < 0 || K <= 0 || (K % 64) != 0 || ldy < N) return NVFP4_ERR_SHAPE;
     if (M >= (1ll << 31) - 256 || N >= (1ll << 31) - 256 || K >= (1ll << 31)) return NVFP4_ERR_SHAPE;
@@ -615,7 +640,8 @@ nvfp4_status linear_impl(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const 
     st = check_arch(info);
     if (st != NVFP4_OK) return st;
 
-    const int bn = choose_variant(M, N);
+    int bn = choose_variant(M, N);
+    if (fused != nullptr && bn == 128) bn = 256;          // the fused epilogue pairs 32 columns: 256-wide tiles only
     const int tile_n = bn == 128 ? 128 : 256;
     GemmMaps tm;
     std::memset(&tm, 0, sizeof(tm));
@@ -632,7 +658,7 @@ nvfp4_status linear_impl(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const 
 
     GemmParams p;
     std::memset(&p, 0, sizeof(p));
-    if ((flags & NVFP4_OUT_F32) == 0u && aligned16(d_y) && (ldy % 8) == 0) {
+    if (fused == nullptr && (flags & NVFP4_OUT_F32) == 0u && aligned16(d_y) && (ldy % 8) == 0) {
         st = output_tensor_map(d_y, M, N, ldy, &tm.y);
         if (st != NVFP4_OK) return st;
         p.tma_store = 1u;
@@ -674,6 +700,21 @@ nvfp4_status linear_impl(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const 
     }
     cudaStream_t s = as_stream(stream);
     const bool fullk = (K % 256) == 0;
+    if (fused != nullptr) {
+        p.g_h = fused->g_h;
+        p.h_codes = fused->h_codes;
+        p.h_sf = fused->h_sf;
+        p.h_katoms = fused->h_katoms;
+        p.inner = fused->inner;
+        p.dbg_y = fused->dbg_y;
+        p.dbg_h = fused->dbg_h;
+        p.split_k = 1;
+        p.k_per_split = p.k_tiles;
+        if (bn == 2) return fullk ? launch_gemm<256, 5, true, true, kEpiSwiglu>(tm, p, info.sm_count, s)
+                                  : launch_gemm<256, 5, true, false, kEpiSwiglu>(tm, p, info.sm_count, s);
+        return fullk ? launch_gemm<256, 3, false, true, kEpiSwiglu>(tm, p, info.sm_count, s)
+                     : launch_gemm<256, 3, false, false, kEpiSwiglu>(tm, p, info.sm_count, s);
+    }
     switch (bn) {
         case 128: return fullk ? launch_gemm<128, 5, false, true>(tm, p, info.sm_count, s) : launch_gemm<128, 5, false, false>(tm, p, info.sm_count, s);
         case 256: return fullk ? launch_gemm<256, 3, false, true>(tm, p, info.sm_count, s) : launch_gemm<256, 3, false, false>(tm, p, info.sm_count, s);
@@ -794,6 +835,29 @@ nvfp4_status nvfp4_linear(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const
     }
     return linear_impl(d_a_codes, d_a_sf, d_g_a, M, K, d_w_codes, d_w_sf, N, segs, d_g_seg, nseg, d_y, ldy, flags,
                        d_workspace, workspace_bytes, split, split_bytes, stream);
+}
+
+nvfp4_status nvfp4_linear_swiglu(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const float* d_g_a, int64_t M, int64_t K,
+                                 const uint8_t* d_w_codes, const uint8_t* d_w_sf, int64_t inner, const float* d_g_gate_up,
+                                 const float* d_g_h, uint8_t* d_h_codes, uint8_t* d_h_sf, void* d_dbg_y, void* d_dbg_h,
+                                 void* d_workspace, size_t workspace_bytes, void* stream) {
+    if (d_g_h == nullptr || d_h_codes == nullptr || d_h_sf == nullptr) return NVFP4_ERR_NULL;
+    if (inner <= 0 || (inner % 64) != 0 || inner >= (1ll << 29)) return NVFP4_ERR_SHAPE;
+    if (!aligned16(d_h_codes) || (reinterpret_cast<uintptr_t>(d_h_sf) & 3u) != 0 ||
+        ((reinterpret_cast<uintptr_t>(d_dbg_y) | reinterpret_cast<uintptr_t>(d_dbg_h)) & 31u) != 0)
+        return NVFP4_ERR_ALIGN;
+    GemmParams fused;
+    std::memset(&fused, 0, sizeof(fused));
+    fused.g_h = d_g_h;
+    fused.h_codes = d_h_codes;
+    fused.h_sf = d_h_sf;
+    fused.h_katoms = static_cast<int32_t>(inner / 64);
+    fused.inner = static_cast<int32_t>(inner);
+    fused.dbg_y = d_dbg_y;
+    fused.dbg_h = d_dbg_h;
+    const nvfp4_segment segs[2] = {{0, inner}, {inner, inner}};        // only their scales are used: columns are interleaved
+    return linear_impl(d_a_codes, d_a_sf, d_g_a, M, K, d_w_codes, d_w_sf, 2 * inner, segs, d_g_gate_up, 2, nullptr, 2 * inner, 0u,
+                       d_workspace, workspace_bytes, nullptr, 0, stream, 0, &fused);
 }
 
 size_t nvfp4_linear_bf16_workspace_bytes(int64_t M, int64_t N, int64_t K, int nseg) {

@@ -20,7 +20,19 @@ namespace nvfp4 {
 struct SegTable {
     int32_t nseg;                          // 0: a single global scale g[0]
     int32_t row_end[NVFP4_MAX_SEGMENTS];   // exclusive end row of each segment (ascending)
+    int32_t il_inner;                      // > 0: the tensor is [gate rows 0..inner) | up rows 0..inner)] and is written
+                                           // with its rows interleaved 16 by 16 (see il_row)
 };
+
+// Output row of input row r when gate and up rows are interleaved in groups of 16: output rows
+// 32 b .. 32 b + 15 are gate rows 16 b .. 16 b + 15, rows 32 b + 16 .. 32 b + 31 the matching up rows.
+// A GEMM against weights in this order produces, per 32 output columns, the 16 gate and the 16 up
+// values of one 16-element block of h = silu(gate) * up.
+__device__ __forceinline__ int32_t il_row(int32_t r, int32_t inner) {
+    const int32_t up = r >= inner ? 1 : 0;
+    const int32_t q = r - up * inner;
+    return (q >> 4) * 32 + up * 16 + (q & 15);
+}
 
 __device__ __forceinline__ int seg_of(const SegTable& t, int32_t row) {
     int s = 0;
@@ -124,19 +136,19 @@ __device__ __forceinline__ uint2 quantize_block(const uint32_t (&v)[8], float g,
     return out;
 }
 
-// silu(g) * u = g * sigmoid(g) * u in binary32 with the hardware's approximate exp2 and
-// reciprocal (2 MUFU + 6 arithmetic instructions per element).  With z = exp(-|g|) in (0, 1]:
-// sigmoid(g) = 1 / (1 + z) for g >= 0 and z / (1 + z) for g < 0, so nothing overflows and very
-// negative gates keep their (tiny, possibly subnormal) value.  The relative error before the bf16
-// rounding is a few 2^-22 (the exponent's rounding adds |g| * 2^-24 * ln 2 for large |g|), so the
-// rounded result equals the correctly rounded definition except in about one case in 10^4 and is
-// never more than one bf16 ulp away.
+// silu(g) * u = g / (1 + exp(-g)) * u in binary32 with the hardware's approximate exp2 and
+// reciprocal (2 MUFU + 4 arithmetic instructions per element).  The relative error before the
+// bf16 rounding is a few 2^-22 (the exponent's rounding adds |g| * 2^-24 * ln 2 for large |g|),
+// so the rounded result equals the correctly rounded definition except in about one case in
+// 10^4 and is never more than one bf16 ulp away -- down to magnitudes of about 2^-100: for
+// g < -88 exp2 overflows to +inf and the result is a zero of the right sign where the definition
+// gives |g| e^g |u| < 1e-36 |u| (no NVFP4 block can hold such a value next to anything else; the
+// sign, which the codes keep, is right).  For g > 126 exp2 flushes to 0 and the result is g * u.
 __device__ __forceinline__ float silu_mul(float g, float u) {
-    float z, r;
-    asm("ex2.approx.f32 %0, %1;" : "=f"(z) : "f"(__fmul_rn(fabsf(g), -1.44269504088896341f)));
-    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(__fadd_rn(1.0f, z)));
-    const float sig = g >= 0.0f ? r : __fmul_rn(z, r);
-    return __fmul_rn(__fmul_rn(g, sig), u);
+    float e, r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(__fmul_rn(g, -1.44269504088896341f)));
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(__fadd_rn(1.0f, e)));
+    return __fmul_rn(__fmul_rn(g, r), u);
 }
 
 // 16 gate values and 16 up values (packed bf16) -> 16 values of bf16(silu(gate) * up), packed
@@ -212,12 +224,13 @@ quantize_kernel(const uint16_t* __restrict__ x, int32_t M, int32_t K, int64_t ld
             c1 = __fdiv_rn(1.0f, __fmul_rn(6.0f, g));
         }
         const uint16_t* xrow = x + static_cast<int64_t>(row) * ld;
-        uint8_t* crow = codes + static_cast<int64_t>(row) * (K >> 1);
+        const int32_t orow = segs.il_inner > 0 ? il_row(row, segs.il_inner) : row;      // where this row is written
+        uint8_t* crow = codes + static_cast<int64_t>(orow) * (K >> 1);
         // scale bytes of this row: byte offset of block kb is sf_row + (kb >> 2) * 512 + (kb & 3)
         // in the tensor-core layout, sf_row + kb in the linear one
         uint8_t* sf_row = MMA_LAYOUT
-            ? sf + static_cast<int64_t>(row >> 7) * katoms * 512 + (row & 31) * 16 + ((row & 127) >> 5) * 4
-            : sf + static_cast<int64_t>(row) * KB;
+            ? sf + static_cast<int64_t>(orow >> 7) * katoms * 512 + (orow & 31) * 16 + ((orow & 127) >> 5) * 4
+            : sf + static_cast<int64_t>(orow) * KB;
         float rstd = 0.0f;
         if (MODE == kQuantRmsnorm) {
             float ss = 0.0f;
