@@ -463,7 +463,10 @@ def run_gpu(args):
         achieved = wl.flops / (gemm_ms * 1e-3) / 1e12
         quant_in_step_gbs = None
     fp4_peak, peak_basis = tensor_peak(peaks, total_ms * 1e-3, clocks)
-    clock_scaled = (148 * 32768 * clocks["sm_mhz"] * 1e6 / 1e12) if clocks.get("sm_mhz") else None
+    # the SM clock the last GEMM of the timed region really ran at, from the kernel's own counters
+    # (the management library's samples lag: they still show the idle boost clock after 20 ms of load)
+    kernel_mhz, _ = nv.last_gemm_clock(ws if args.workload == "mlp" else wss[(counter[0] - 1) % nset])
+    clock_scaled = (148 * 32768 * kernel_mhz * 1e6 / 1e12) if kernel_mhz > 0 else None
     roofline = {"kernel": "gemm_kernel (tcgen05 block-scaled FP4)", "bound": "tensor",
                 "achieved": round(achieved, 2), "peak": round(fp4_peak, 1), "unit": "TFLOP/s",
                 "frac": round(achieved / fp4_peak, 4), "peak_basis": peak_basis,
@@ -471,7 +474,8 @@ def run_gpu(args):
                 "frac_of_sustained_x4": round(achieved / (peaks["bf16_tflops_sustained"] * FP4_OVER_BF16), 4),
                 "frac_of_nominal_9pf": round(achieved / NOMINAL_FP4_TFLOPS, 4),
                 "frac_of_clock_scaled_peak": None if not clock_scaled else round(achieved / clock_scaled, 4),
-                "clock_scaled_peak_basis": "148 SMs x 32768 FLOP/clk x median SM clock during the timed region",
+                "sm_mhz_in_kernel": round(kernel_mhz, 1),
+                "clock_scaled_peak_basis": "148 SMs x 32768 FLOP/clk x the SM clock read inside the last GEMM of the timed region (cycle counter / wall clock)",
                 "avg_launch_ms": round(gemm_ms, 4),
                 "traffic": ncu_traffic("gemm_kernel")}
     result["roofline"] = roofline

@@ -358,6 +358,14 @@ nvfp4_status nvfp4_workspace_reset(void* d_workspace, size_t workspace_bytes, vo
 nvfp4_status nvfp4_device_status(const void* d_workspace, void* stream);
 
 /*
+ * Measurement aid: the SM clock the last tensor-core GEMM launched on this workspace really ran at
+ * (its first CTA's cycle counter over the wall clock, both read inside the kernel and left in the
+ * status block), and that CTA's lifetime in microseconds.  Under a power cap the clock drops within
+ * microseconds, long before a management-library sample shows it.  Synchronises `stream`.
+ */
+nvfp4_status nvfp4_last_gemm_clock(const void* d_workspace, double* sm_mhz, double* kernel_us, void* stream);
+
+/*
  * Time limit of every wait inside the GEMM kernel, in nanoseconds (0 restores the default of
  * 2 s).  A CTA whose wait runs out stops issuing work, lets what it has in flight finish, frees
  * its tensor memory and raises NVFP4_ERR_TIMEOUT in the workspace status word; the kernel

@@ -28,7 +28,7 @@ EXPORTS = (
     "nvfp4_quantize_weight", "nvfp4_quantize_weight_gate_up", "nvfp4_linear_swiglu",
     "nvfp4_harmonize_scales", "nvfp4_tensor_stats", "nvfp4_linear", "nvfp4_linear_workspace_bytes", "nvfp4_linear_bf16",
     "nvfp4_linear_bf16_workspace_bytes", "nvfp4_linear_bf16_static", "nvfp4_static_status", "nvfp4_workspace_reset", "nvfp4_device_status",
-    "nvfp4_set_wait_limit_ns", "nvfp4_selftest_bounded_wait", "nvfp4_launch_count", "nvfp4_set_gemm_variant", "nvfp4_gemm_variants", "nvfp4_status_string",
+    "nvfp4_last_gemm_clock", "nvfp4_set_wait_limit_ns", "nvfp4_selftest_bounded_wait", "nvfp4_launch_count", "nvfp4_set_gemm_variant", "nvfp4_gemm_variants", "nvfp4_status_string",
 )
 
 
@@ -91,6 +91,8 @@ def lib() -> ctypes.CDLL:
     L.nvfp4_workspace_reset.argtypes = [vp, sz, vp]
     L.nvfp4_device_status.restype = i32
     L.nvfp4_device_status.argtypes = [vp, vp]
+    L.nvfp4_last_gemm_clock.restype = i32
+    L.nvfp4_last_gemm_clock.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double), vp]
     L.nvfp4_set_wait_limit_ns.restype = i32
     L.nvfp4_set_wait_limit_ns.argtypes = [ctypes.c_uint64]
     L.nvfp4_selftest_bounded_wait.restype = i32
@@ -351,6 +353,15 @@ def static_status(stream=None) -> int:
     """Status word of the library's static scratch (synchronises the stream); a failure also
     clears the word and re-zeroes the split-K part of the array."""
     return int(lib().nvfp4_static_status(_stream(stream)))
+
+
+def last_gemm_clock(workspace: torch.Tensor, stream=None) -> Tuple[float, float]:
+    """(SM clock in MHz, lifetime in us) of the first CTA of the last tensor-core GEMM launched on this
+    workspace, from the kernel's own cycle counter and wall clock.  Synchronises the stream."""
+    mhz, us = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    _check(lib().nvfp4_last_gemm_clock(_ptr(workspace), ctypes.byref(mhz), ctypes.byref(us), _stream(stream)),
+           "nvfp4_last_gemm_clock")
+    return mhz.value, us.value
 
 
 def workspace_reset(workspace: torch.Tensor, stream=None) -> None:

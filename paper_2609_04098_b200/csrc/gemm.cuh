@@ -183,6 +183,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     if (PAIR) ptx::cluster_sync_all(); else __syncthreads();   // barriers and TMEM exist from here on
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // CTA 0 leaves its own clock readings in the status block (words 2..9: cycle counter and wall clock
+    // at start and end), so that the host can tell at which SM clock the kernel really ran -- under a
+    // power cap the clock drops within microseconds, long before a management-library sample shows it
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        reinterpret_cast<unsigned long long*>(p.status)[1] = static_cast<unsigned long long>(clock64());
+        reinterpret_cast<unsigned long long*>(p.status)[2] = ptx::globaltimer_ns();
+    }
     // Everything above ran while the kernel in front of this one (the activation quantizer, which
     // releases its dependents early) may still have been working; nothing below may read global
     // memory before that kernel has finished.
@@ -391,10 +398,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 }
                 areg[i] = a;
             }
-            // one lane polls, with a back-off: 128 threads spinning on the barrier would take
-            // shared-memory cycles away from the MMAs for the whole main loop
+            // one lane polls (try_wait suspends the thread in hardware between looks): 128 threads
+            // spinning on the barrier would take shared-memory cycles away from the MMAs
             bool ok = true;
-            if (lane == 0) ok = ptx::mbar_wait_bounded(&tfull[acc], aph, abort_flag, p.wait_limit_ns, peer_abort, 128u);
+            if (lane == 0) ok = ptx::mbar_wait_bounded(&tfull[acc], aph, abort_flag, p.wait_limit_ns, peer_abort);
             ok = __shfl_sync(0xffffffffu, static_cast<int>(ok), 0) != 0;
             if (!ok) break;
             ptx::tc_fence_after();
@@ -639,6 +646,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         if (PAIR) ptx::tmem_dealloc_pair(tmem_base, kTmemCols); else ptx::tmem_dealloc(tmem_base, kTmemCols);
     }
     if (threadIdx.x == 0 && *abort_flag != 0u) atomicExch(p.status, static_cast<uint32_t>(NVFP4_ERR_TIMEOUT));
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        reinterpret_cast<unsigned long long*>(p.status)[3] = static_cast<unsigned long long>(clock64());
+        reinterpret_cast<unsigned long long*>(p.status)[4] = ptx::globaltimer_ns();
+    }
 }
 
 }  // namespace nvfp4

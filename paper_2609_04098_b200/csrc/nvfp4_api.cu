@@ -284,23 +284,36 @@ nvfp4_status launch_quantize(const uint16_t* x, int64_t M, int64_t K, int64_t ld
     const int64_t max_blocks = static_cast<int64_t>(sm_count) * per_sm;
     if (blocks > max_blocks) blocks = max_blocks;
     if (blocks < 1) blocks = 1;
-    quantize_kernel<MMA, kUnroll, MODE><<<static_cast<int>(blocks), 256, 0, stream>>>(
-        x, static_cast<int32_t>(M), static_cast<int32_t>(K), ld, d_g, segs, aux, eps, d_codes, d_sf, h_out,
-        static_cast<int32_t>(chunks), static_cast<int32_t>(per_unit), static_cast<int32_t>(units_per_row),
-        static_cast<int32_t>(units));
+    // launched so that it may start while the kernel in front of it drains (if that kernel says so, as
+    // this one does for its own dependents); its first global read waits for that kernel's completion
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof(cfg));
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.gridDim = dim3(static_cast<unsigned>(blocks), 1, 1);
+    cfg.blockDim = dim3(256, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t le = cudaLaunchKernelEx(&cfg, quantize_kernel<MMA, kUnroll, MODE>, x, static_cast<int32_t>(M),
+                                              static_cast<int32_t>(K), ld, d_g, segs, aux, eps, d_codes, d_sf, h_out,
+                                              static_cast<int32_t>(chunks), static_cast<int32_t>(per_unit),
+                                              static_cast<int32_t>(units_per_row), static_cast<int32_t>(units));
     g_launches.fetch_add(1, std::memory_order_relaxed);
-    return cudaGetLastError() == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+    return le == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
 
-// RMSNorm -> quantize with the row held in registers by W warps (rows of up to 8 * kRmsChunks chunks)
-template <bool MMA, int W>
+// RMSNorm -> quantize with the row held in registers by W warps of NCH chunks each
+template <bool MMA, int W, int NCH>
 nvfp4_status launch_rmsnorm(const uint16_t* x, int64_t M, int64_t rows_total, int64_t K, int64_t ld, const float* d_g,
                             const uint16_t* gain, float eps, uint8_t* d_codes, uint8_t* d_sf, uint16_t* y_out,
                             int64_t chunks, int sm_count, cudaStream_t stream) {
     static std::atomic<int> per_sm_cache{0};
     int per_sm = per_sm_cache.load(std::memory_order_relaxed);
     if (per_sm == 0) {
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rmsnorm_quantize_kernel<MMA, W>, 256, 0) != cudaSuccess ||
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rmsnorm_quantize_kernel<MMA, W, NCH>, 256, 0) != cudaSuccess ||
             per_sm < 1) {
             cudaGetLastError();
             per_sm = 2;
@@ -312,7 +325,7 @@ nvfp4_status launch_rmsnorm(const uint16_t* x, int64_t M, int64_t rows_total, in
     const int64_t max_blocks = static_cast<int64_t>(sm_count) * per_sm;
     if (blocks > max_blocks) blocks = max_blocks;
     if (blocks < 1) blocks = 1;
-    rmsnorm_quantize_kernel<MMA, W><<<static_cast<int>(blocks), 256, 0, stream>>>(
+    rmsnorm_quantize_kernel<MMA, W, NCH><<<static_cast<int>(blocks), 256, 0, stream>>>(
         x, static_cast<int32_t>(M), static_cast<int32_t>(rows_total), static_cast<int32_t>(K), ld, d_g, gain, eps,
         d_codes, d_sf, y_out, static_cast<int32_t>(chunks), static_cast<int32_t>((chunks + W - 1) / W));
     g_launches.fetch_add(1, std::memory_order_relaxed);
@@ -325,20 +338,20 @@ nvfp4_status quantize_impl(const void* d_x, int64_t M, int64_t K, int64_t ld, co
                            const uint16_t* aux = nullptr, float eps = 0.0f, uint16_t* h_out = nullptr) {
     const int64_t chunks = (K + 511) / 512;              // 512 elements = one block per lane
     if (M >= (1ll << 31) || K >= (1ll << 31)) return NVFP4_ERR_SHAPE;
-    if (mode == kQuantRmsnorm && chunks <= 8 * kRmsChunks) {
+    if (mode == kQuantRmsnorm && chunks <= 8 * kRmsChunksMax) {
         const uint16_t* xr = reinterpret_cast<const uint16_t*>(d_x);
         const int64_t rows_all = (layout == NVFP4_SF_MMA) ? (M + 127) / 128 * 128 : M;
         const bool mma_l = layout == NVFP4_SF_MMA;
+        // fewest warps per row that keep a warp's share at kRmsChunksMax chunks
         int w = 1;
-        while (w < 8 && (chunks + w - 1) / w > kRmsChunks) w *= 2;
-        if (w == 1 && chunks >= 2 && chunks % 2 == 0) w = 2;       // shorter dependency chain per row, same registers
-#define NVFP4_LAUNCH_R(MMA_, W_) \
-    launch_rmsnorm<MMA_, W_>(xr, M, rows_all, K, ld, d_g, aux, eps, d_codes, d_sf, h_out, chunks, info.sm_count, stream)
+        while (w < 8 && (chunks + w - 1) / w > kRmsChunksMax) w *= 2;
+#define NVFP4_LAUNCH_R(MMA_, W_, NCH_) \
+    launch_rmsnorm<MMA_, W_, NCH_>(xr, M, rows_all, K, ld, d_g, aux, eps, d_codes, d_sf, h_out, chunks, info.sm_count, stream)
         switch (w) {
-            case 1: return mma_l ? NVFP4_LAUNCH_R(true, 1) : NVFP4_LAUNCH_R(false, 1);
-            case 2: return mma_l ? NVFP4_LAUNCH_R(true, 2) : NVFP4_LAUNCH_R(false, 2);
-            case 4: return mma_l ? NVFP4_LAUNCH_R(true, 4) : NVFP4_LAUNCH_R(false, 4);
-            default: return mma_l ? NVFP4_LAUNCH_R(true, 8) : NVFP4_LAUNCH_R(false, 8);
+            case 1: return mma_l ? NVFP4_LAUNCH_R(true, 1, 5) : NVFP4_LAUNCH_R(false, 1, 5);
+            case 2: return mma_l ? NVFP4_LAUNCH_R(true, 2, 5) : NVFP4_LAUNCH_R(false, 2, 5);
+            case 4: return mma_l ? NVFP4_LAUNCH_R(true, 4, 5) : NVFP4_LAUNCH_R(false, 4, 5);
+            default: return mma_l ? NVFP4_LAUNCH_R(true, 8, 5) : NVFP4_LAUNCH_R(false, 8, 5);
         }
 #undef NVFP4_LAUNCH_R
     }
@@ -940,6 +953,17 @@ nvfp4_status nvfp4_device_status(const void* d_workspace, void* stream) {
     if (word == NVFP4_ERR_TIMEOUT) return NVFP4_ERR_TIMEOUT;
     if (word == NVFP4_ERR_SCALE) return NVFP4_ERR_SCALE;
     return NVFP4_ERR_CUDA;
+}
+
+nvfp4_status nvfp4_last_gemm_clock(const void* d_workspace, double* sm_mhz, double* kernel_us, void* stream) {
+    if (d_workspace == nullptr || sm_mhz == nullptr || kernel_us == nullptr) return NVFP4_ERR_NULL;
+    unsigned long long w[5] = {0, 0, 0, 0, 0};
+    if (cudaMemcpyAsync(w, d_workspace, sizeof(w), cudaMemcpyDeviceToHost, as_stream(stream)) != cudaSuccess) return NVFP4_ERR_CUDA;
+    if (cudaStreamSynchronize(as_stream(stream)) != cudaSuccess) return NVFP4_ERR_CUDA;
+    const double ns = static_cast<double>(w[4] - w[2]), cycles = static_cast<double>(w[3] - w[1]);
+    *kernel_us = ns * 1e-3;
+    *sm_mhz = ns > 0.0 ? cycles / ns * 1e3 : 0.0;
+    return NVFP4_OK;
 }
 
 namespace nvfp4 {

@@ -189,14 +189,17 @@ quantize_kernel(const uint16_t* __restrict__ x, int32_t M, int32_t K, int64_t ld
                 const float* __restrict__ g_ptr, SegTable segs, const uint16_t* __restrict__ aux, float eps,
                 uint8_t* __restrict__ codes, uint8_t* __restrict__ sf, uint16_t* __restrict__ h_out,
                 int32_t chunks_per_row, int32_t chunks_per_unit, int32_t units_per_row, int32_t total_units) {
-    // the GEMM that consumes this tensor may start its prologue and its weight loads now; it
-    // waits for this kernel's completion before it touches the codes and scales written here
+    // the kernel behind this one (the GEMM that consumes this tensor, or the next quantizer) may start
+    // its prologue now; it waits for this kernel's completion before it reads anything
     ptx::pdl_launch_dependents();
     const int lane = threadIdx.x & 31;
     const int32_t warp_global = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int32_t nwarps = gridDim.x * (blockDim.x >> 5);
     const int32_t KB = K >> 4;
     const int32_t katoms = (KB + 3) >> 2;
+    // this kernel itself may have been started early: everything it reads (the tensor, the global scale)
+    // may come from the kernel in front of it
+    ptx::pdl_wait();
     const float g_single = (segs.nseg == 0) ? __ldg(g_ptr) : 0.0f;
     const float c1_single = __fdiv_rn(1.0f, __fmul_rn(6.0f, g_single));
 
@@ -316,19 +319,21 @@ quantize_kernel(const uint16_t* __restrict__ x, int32_t M, int32_t K, int64_t ld
 }
 
 // ------------------------------------------------------------------ RMSNorm -> quantize, row in registers
-// A row is shared by W warps of one CTA (W = 1, 2, 4 or 8; each warp owns up to kRmsChunks
-// consecutive 512-element chunks and each lane one 16-element block per chunk), so the row is read
+// A row is shared by W warps of one CTA (W = 1, 2, 4 or 8; each warp owns up to NCH consecutive
+// 512-element chunks and each lane one 16-element block per chunk), so the row is read
 // from HBM exactly once and stays in registers between the reduction and the quantization:
 //   1. every lane loads its blocks (streaming loads, all in flight at once) and sums their squares;
 //   2. warp butterfly, then the W partial sums meet in shared memory (one named barrier per row;
 //      the two buffers alternate so that no second barrier is needed);
 //   3. y = bf16((x * rstd) * w) per element, then the block is quantized as everywhere else.
 // Rows are dealt round-robin to the row groups of a persistent grid.  Rows M .. M_pad-1 (tensor-core
-// layout only) get zero scales.
-constexpr int kRmsChunks = 5;
+// layout only) get zero scales.  (Three chunks per warp at three CTAs per SM measured no faster than
+// five chunks at two: the kernel is bound by its instruction count -- square, normalise, scale and
+// round on top of the quantizer's own work -- not by the loads it has in flight.)
+constexpr int kRmsChunksMax = 5;
 
-template <bool MMA_LAYOUT, int W>
-__global__ void __launch_bounds__(256, 2)
+template <bool MMA_LAYOUT, int W, int NCH>
+__global__ void __launch_bounds__(256, NCH <= 3 ? 3 : 2)
 rmsnorm_quantize_kernel(const uint16_t* __restrict__ x, int32_t M, int32_t rows_total, int32_t K, int64_t ld,
                         const float* __restrict__ g_ptr, const uint16_t* __restrict__ gain, float eps,
                         uint8_t* __restrict__ codes, uint8_t* __restrict__ sf, uint16_t* __restrict__ y_out,
@@ -359,9 +364,9 @@ rmsnorm_quantize_kernel(const uint16_t* __restrict__ x, int32_t M, int32_t rows_
             continue;                                           // a whole group skips together: no barrier is missed
         }
         const uint16_t* xrow = x + static_cast<int64_t>(row) * ld;
-        uint32_t v[kRmsChunks][8];
+        uint32_t v[NCH][8];
 #pragma unroll
-        for (int i = 0; i < kRmsChunks; ++i) {
+        for (int i = 0; i < NCH; ++i) {
             const int32_t col = (c_begin + i) * 512 + lane * 16;
             if (c_begin + i < c_end && col < K) {
                 ldg256_stream(xrow + col, v[i]);
@@ -372,7 +377,7 @@ rmsnorm_quantize_kernel(const uint16_t* __restrict__ x, int32_t M, int32_t rows_
         }
         float ss = 0.0f;
 #pragma unroll
-        for (int i = 0; i < kRmsChunks; ++i) {
+        for (int i = 0; i < NCH; ++i) {
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
                 const float lo = __uint_as_float(v[i][e] << 16), hi = __uint_as_float(v[i][e] & 0xFFFF0000u);
@@ -393,7 +398,7 @@ rmsnorm_quantize_kernel(const uint16_t* __restrict__ x, int32_t M, int32_t rows_
         const float rstd = __frcp_rn(__fsqrt_rn(__fadd_rn(__fdiv_rn(ss, static_cast<float>(K)), eps)));
         uint8_t* crow = codes + static_cast<int64_t>(row) * (K >> 1);
 #pragma unroll
-        for (int i = 0; i < kRmsChunks; ++i) {
+        for (int i = 0; i < NCH; ++i) {
             if (c_begin + i >= c_end) break;                    // warp-uniform
             const int32_t col = (c_begin + i) * 512 + lane * 16;
             const bool in_range = col < K;
