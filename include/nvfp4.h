@@ -358,6 +358,31 @@ nvfp4_status nvfp4_workspace_reset(void* d_workspace, size_t workspace_bytes, vo
 nvfp4_status nvfp4_device_status(const void* d_workspace, void* stream);
 
 /*
+ * Gated delta-rule recurrence, clean and perturbed trajectory in lockstep (paper: Background, Eq. 1-2;
+ * Section 5.3 and Appendix "Error propagation": one clean FP32 trajectory and perturbed ones on
+ * identical inputs, state error over time).  Per value head h, with K = V = 128, in binary32:
+ *     g_t = -exp(A_log[h]) * softplus(a_t + dt_bias[h]);  alpha_t = exp(g_t);  beta_t = sigmoid(b_t)
+ *     S_t = alpha_t S_{t-1} + beta_t k_t (v_t - S_{t-1}^T k_t)^T;   o_t = S_t^T (q_t / sqrt(128));   S_0 = 0
+ * run once on (q, k, v, a, b) and once on (q2, k2, v2, a2, b2) -- the same projections computed another
+ * way, e.g. through the NVFP4 layer -- and compared every `sample_every` tokens:
+ *     rel_state[s, h] = ||S2 - S||_F / ||S||_F,   rel_out[s, h] = ||o2 - o|| / ||o||   at token (s+1)*sample_every - 1
+ *   d_q, d_k    float [T, Hk, 128], l2-normalised per head (the caller's job);  d_v float [T, Hv, 128]
+ *   d_a, d_b    float [T, Hv] gate pre-activations;  d_A_log, d_dt_bias float [Hv]
+ *   Hv % Hk == 0: value head h reads query/key head h / (Hv / Hk)
+ *   impulse_step >= 0: after that token the second trajectory's state is scaled by (1 + impulse_rel), once
+ *                      (the paper's one-off state perturbation); < 0: none
+ *   d_rel_state, d_rel_out   out float [T / sample_every, Hv]
+ *   d_final_state            optional (may be NULL) out float [2, Hv, 128 (k), 128 (v)]
+ * Any second-trajectory pointer may equal its clean counterpart.  Errors: NULL, T < 0, Hv % Hk != 0,
+ * sample_every < 1, impulse_rel <= -1.
+ */
+nvfp4_status nvfp4_gdn_lockstep(const float* d_q, const float* d_k, const float* d_v, const float* d_a, const float* d_b,
+                                const float* d_q2, const float* d_k2, const float* d_v2, const float* d_a2, const float* d_b2,
+                                const float* d_A_log, const float* d_dt_bias, int64_t T, int Hk, int Hv,
+                                int64_t impulse_step, float impulse_rel, int64_t sample_every,
+                                float* d_rel_state, float* d_rel_out, float* d_final_state, void* stream);
+
+/*
  * Measurement aid: the SM clock the last tensor-core GEMM launched on this workspace really ran at
  * (its first CTA's cycle counter over the wall clock, both read inside the kernel and left in the
  * status block), and that CTA's lifetime in microseconds.  Under a power cap the clock drops within

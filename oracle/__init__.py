@@ -299,3 +299,55 @@ def gemm(a_codes, a_sf, g_a, w_codes, w_sf, g_col, rows=None, cols=None) -> np.n
     if rc != 0:
         raise RuntimeError("oracle gemm failed (%d)" % rc)
     return out
+
+
+# -- gated delta-rule recurrence (paper: Background, Eq. 1-2; Section 5.3 lockstep study) ------------
+def gdn_gates(a: np.ndarray, b: np.ndarray, A_log: np.ndarray, dt_bias: np.ndarray):
+    """Eq. 1: g = -exp(A_log) * softplus(a + dt_bias); alpha = exp(g) in (0, 1); beta = sigmoid(b)."""
+    a = np.asarray(a, np.float64)
+    z = a + np.asarray(dt_bias, np.float64)
+    softplus = np.logaddexp(0.0, z)
+    alpha = np.exp(-np.exp(np.asarray(A_log, np.float64)) * softplus)
+    bb = np.asarray(b, np.float64)
+    e = np.exp(-np.abs(bb))                                    # sigmoid without overflow: e in (0, 1]
+    beta = np.where(bb >= 0, 1.0 / (1.0 + e), e / (1.0 + e))
+    return alpha, beta
+
+
+def gdn_recurrence(q, k, v, a, b, A_log, dt_bias, impulse_step: int = -1, impulse_rel: float = 0.0):
+    """Eq. 2 in float64, token by token: S_t = alpha_t S_{t-1} + beta_t k_t (v_t - S_{t-1}^T k_t)^T and
+    o_t = S_t^T (q_t / sqrt(K)), S_0 = 0.  q, k: [T, Hk, K]; v: [T, Hv, V]; a, b: [T, Hv]; value head h
+    reads query/key head h // (Hv // Hk).  Returns (states [T, Hv, K, V], outputs [T, Hv, V]).
+    `impulse_step` >= 0 scales the state by (1 + impulse_rel) once, after that token."""
+    q, k, v = (np.asarray(t, np.float64) for t in (q, k, v))
+    T, Hk, K = q.shape
+    Hv, V = v.shape[1], v.shape[2]
+    alpha, beta = gdn_gates(a, b, A_log, dt_bias)
+    rep = Hv // Hk
+    S = np.zeros((Hv, K, V))
+    states = np.empty((T, Hv, K, V))
+    outs = np.empty((T, Hv, V))
+    for t in range(T):
+        for h in range(Hv):
+            kt, qt = k[t, h // rep], q[t, h // rep]
+            pred = S[h].T @ kt                                   # what the state predicts for this key
+            S[h] = alpha[t, h] * S[h] + beta[t, h] * np.outer(kt, v[t, h] - pred)
+            outs[t, h] = S[h].T @ (qt / np.sqrt(K))
+            if t == impulse_step:
+                S[h] = S[h] * (1.0 + impulse_rel)
+        states[t] = S
+    return states, outs
+
+
+def gdn_lockstep(clean, other, A_log, dt_bias, sample_every: int, impulse_step: int = -1, impulse_rel: float = 0.0):
+    """Clean and second trajectory on their own inputs; relative state and output error at the sampled
+    tokens (sample_every - 1, 2 * sample_every - 1, ...): ([ns, Hv], [ns, Hv])."""
+    S0, o0 = gdn_recurrence(*clean, A_log, dt_bias)
+    S1, o1 = gdn_recurrence(*other, A_log, dt_bias, impulse_step, impulse_rel)
+    idx = np.arange(sample_every - 1, S0.shape[0], sample_every)
+    ds = np.sqrt(((S1[idx] - S0[idx]) ** 2).sum(axis=(2, 3)))
+    rs = np.sqrt((S0[idx] ** 2).sum(axis=(2, 3)))
+    do = np.sqrt(((o1[idx] - o0[idx]) ** 2).sum(axis=2))
+    ro = np.sqrt((o0[idx] ** 2).sum(axis=2))
+    with np.errstate(divide="ignore", invalid="ignore"):
+        return np.where(rs > 0, ds / rs, 0.0), np.where(ro > 0, do / ro, 0.0)

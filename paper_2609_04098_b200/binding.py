@@ -28,7 +28,7 @@ EXPORTS = (
     "nvfp4_quantize_weight", "nvfp4_quantize_weight_gate_up", "nvfp4_linear_swiglu",
     "nvfp4_harmonize_scales", "nvfp4_tensor_stats", "nvfp4_linear", "nvfp4_linear_workspace_bytes", "nvfp4_linear_bf16",
     "nvfp4_linear_bf16_workspace_bytes", "nvfp4_linear_bf16_static", "nvfp4_static_status", "nvfp4_workspace_reset", "nvfp4_device_status",
-    "nvfp4_last_gemm_clock", "nvfp4_set_wait_limit_ns", "nvfp4_selftest_bounded_wait", "nvfp4_launch_count", "nvfp4_set_gemm_variant", "nvfp4_gemm_variants", "nvfp4_status_string",
+    "nvfp4_gdn_lockstep", "nvfp4_last_gemm_clock", "nvfp4_set_wait_limit_ns", "nvfp4_selftest_bounded_wait", "nvfp4_launch_count", "nvfp4_set_gemm_variant", "nvfp4_gemm_variants", "nvfp4_status_string",
 )
 
 
@@ -91,6 +91,8 @@ def lib() -> ctypes.CDLL:
     L.nvfp4_workspace_reset.argtypes = [vp, sz, vp]
     L.nvfp4_device_status.restype = i32
     L.nvfp4_device_status.argtypes = [vp, vp]
+    L.nvfp4_gdn_lockstep.restype = i32
+    L.nvfp4_gdn_lockstep.argtypes = [vp] * 12 + [i64, i32, i32, i64, ctypes.c_float, i64, vp, vp, vp, vp]
     L.nvfp4_last_gemm_clock.restype = i32
     L.nvfp4_last_gemm_clock.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double), vp]
     L.nvfp4_set_wait_limit_ns.restype = i32
@@ -353,6 +355,26 @@ def static_status(stream=None) -> int:
     """Status word of the library's static scratch (synchronises the stream); a failure also
     clears the word and re-zeroes the split-K part of the array."""
     return int(lib().nvfp4_static_status(_stream(stream)))
+
+
+def nvfp4_gdn_lockstep(clean, other, A_log, dt_bias, sample_every: int, impulse_step: int = -1,
+                       impulse_rel: float = 0.0, final_state: bool = False, stream=None):
+    """Gated delta-rule recurrence on two input sets in lockstep.  ``clean`` and ``other`` are tuples
+    (q [T,Hk,128], k [T,Hk,128], v [T,Hv,128], a [T,Hv], b [T,Hv]) of float32 CUDA tensors.
+    Returns (rel_state [T // sample_every, Hv], rel_out, final states [2,Hv,128,128] or None)."""
+    q, k, v, a, b = clean
+    T, Hk = q.shape[0], q.shape[1]
+    Hv = v.shape[1]
+    for t in tuple(clean) + tuple(other) + (A_log, dt_bias):
+        assert t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()
+    ns = T // sample_every
+    rel_state = torch.zeros((max(ns, 1), Hv), dtype=torch.float32, device=q.device)
+    rel_out = torch.zeros_like(rel_state)
+    fs = torch.empty((2, Hv, 128, 128), dtype=torch.float32, device=q.device) if final_state else None
+    _check(lib().nvfp4_gdn_lockstep(*[_ptr(t) for t in clean], *[_ptr(t) for t in other], _ptr(A_log), _ptr(dt_bias),
+                                    T, Hk, Hv, int(impulse_step), ctypes.c_float(impulse_rel), int(sample_every),
+                                    _ptr(rel_state), _ptr(rel_out), _ptr(fs), _stream(stream)), "nvfp4_gdn_lockstep")
+    return rel_state[:ns], rel_out[:ns], fs
 
 
 def last_gemm_clock(workspace: torch.Tensor, stream=None) -> Tuple[float, float]:

@@ -15,6 +15,7 @@
 #include "decode.cuh"
 #include "gemm.cuh"
 #include "quantize.cuh"
+#include "recurrence.cuh"
 
 namespace nvfp4 {
 namespace {
@@ -953,6 +954,53 @@ nvfp4_status nvfp4_device_status(const void* d_workspace, void* stream) {
     if (word == NVFP4_ERR_TIMEOUT) return NVFP4_ERR_TIMEOUT;
     if (word == NVFP4_ERR_SCALE) return NVFP4_ERR_SCALE;
     return NVFP4_ERR_CUDA;
+}
+
+nvfp4_status nvfp4_gdn_lockstep(const float* d_q, const float* d_k, const float* d_v, const float* d_a, const float* d_b,
+                                const float* d_q2, const float* d_k2, const float* d_v2, const float* d_a2, const float* d_b2,
+                                const float* d_A_log, const float* d_dt_bias, int64_t T, int Hk, int Hv,
+                                int64_t impulse_step, float impulse_rel, int64_t sample_every,
+                                float* d_rel_state, float* d_rel_out, float* d_final_state, void* stream) {
+    if (d_q == nullptr || d_k == nullptr || d_v == nullptr || d_a == nullptr || d_b == nullptr || d_q2 == nullptr ||
+        d_k2 == nullptr || d_v2 == nullptr || d_a2 == nullptr || d_b2 == nullptr || d_A_log == nullptr ||
+        d_dt_bias == nullptr || d_rel_state == nullptr || d_rel_out == nullptr)
+        return NVFP4_ERR_NULL;
+    if (T < 0 || Hk < 1 || Hv < 1 || Hv > 65535 || (Hv % Hk) != 0 || sample_every < 1 || !(impulse_rel > -1.0f)) return NVFP4_ERR_SHAPE;
+    if (T == 0) return NVFP4_OK;
+    DeviceInfo info;
+    nvfp4_status st = check_arch(info);
+    if (st != NVFP4_OK) return st;
+    LockstepParams lp;
+    std::memset(&lp, 0, sizeof(lp));
+    lp.q[0] = d_q; lp.k[0] = d_k; lp.v[0] = d_v; lp.a[0] = d_a; lp.b[0] = d_b;
+    lp.q[1] = d_q2; lp.k[1] = d_k2; lp.v[1] = d_v2; lp.a[1] = d_a2; lp.b[1] = d_b2;
+    lp.A_log = d_A_log;
+    lp.dt_bias = d_dt_bias;
+    lp.T = T;
+    lp.Hk = Hk;
+    lp.Hv = Hv;
+    lp.impulse_step = impulse_step;
+    lp.impulse_rel = impulse_rel;
+    lp.sample_every = sample_every;
+    lp.rel_state = d_rel_state;
+    lp.rel_out = d_rel_out;
+    lp.final_state = d_final_state;
+    const size_t smem = static_cast<size_t>(kGdnDim * (kGdnDim + 1) + kGdnDim) * sizeof(float);
+    static std::mutex mu;
+    static std::unordered_map<int, bool> configured;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        if (!configured[dev]) {
+            if (cudaFuncSetAttribute(gdn_lockstep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
+                return NVFP4_ERR_CUDA;
+            configured[dev] = true;
+        }
+    }
+    gdn_lockstep_kernel<<<Hv, 256, smem, as_stream(stream)>>>(lp);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
 
 nvfp4_status nvfp4_last_gemm_clock(const void* d_workspace, double* sm_mhz, double* kernel_us, void* stream) {
