@@ -75,6 +75,11 @@ typedef enum { NVFP4_SF_LINEAR = 0, NVFP4_SF_MMA = 1 } nvfp4_sf_layout;
                                  since been written by this library only.  Lets decode-sized calls (M <= 256)
                                  split K over several CTAs, which meet in the workspace and leave it zero again.
                                  After NVFP4_ERR_TIMEOUT zero the workspace before the next call with this flag. */
+#define NVFP4_W_RESIDENT 4u   /* caller's promise: the weight operand (codes, scales, global scales) was complete before
+                                 the work in front of this call in the stream was submitted -- true of model weights,
+                                 false of a tensor quantized by the preceding call.  Lets the kernel start fetching
+                                 weights while the kernel in front of it still runs (programmatic dependent launch);
+                                 activations, global scales of activations and outputs are still ordered as usual. */
 
 /*
  * Workspace layout (the same for every entry point and every problem size, so one zero-filled

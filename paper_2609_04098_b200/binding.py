@@ -21,6 +21,7 @@ SF_MMA = 1
 OUT_BF16 = 0
 OUT_F32 = 1
 WS_ZEROED = 2        # workspaces from alloc_workspace are zero-filled, so the binding always promises this
+W_RESIDENT = 4       # the weights were complete before the preceding work of the stream was submitted
 MAX_SEGMENTS = 32
 
 EXPORTS = (
@@ -295,14 +296,16 @@ def alloc_workspace(device, M: int = 0, N: int = 0, K: int = 0, nseg: int = 1, f
 
 
 def nvfp4_linear(a_codes, a_sf, g_a, w_codes, w_sf, segments, g_seg, workspace, out=None,
-                 out_f32: bool = False, stream=None) -> torch.Tensor:
-    """Y[M, N] = (A_q . W_q^T) * g_a * g_seg[segment of n]; bf16 (or float32) output."""
+                 out_f32: bool = False, stream=None, w_resident: bool = False) -> torch.Tensor:
+    """Y[M, N] = (A_q . W_q^T) * g_a * g_seg[segment of n]; bf16 (or float32) output.
+    ``w_resident``: the weights (codes, scales, ``g_seg``) were complete before the work in front of
+    this call was submitted to the stream, so the kernel may fetch them while that work still runs."""
     M, K = a_codes.shape[0], a_codes.shape[1] * 2
     N = w_codes.shape[0]
     pairs = seg_pairs(segments)
     if out is None:
         out = torch.empty((M, N), dtype=torch.float32 if out_f32 else torch.bfloat16, device=a_codes.device)
-    flags = (OUT_F32 if out.dtype == torch.float32 else OUT_BF16) | WS_ZEROED
+    flags = (OUT_F32 if out.dtype == torch.float32 else OUT_BF16) | WS_ZEROED | (W_RESIDENT if w_resident else 0)
     _check(lib().nvfp4_linear(_ptr(a_codes), _ptr(a_sf), _ptr(g_a), M, K, _ptr(w_codes), _ptr(w_sf), N,
                               _segments(pairs), _ptr(g_seg), len(pairs), _ptr(out), out.stride(0), flags,
                               _ptr(workspace), workspace.numel(), _stream(stream)), "nvfp4_linear")
@@ -310,7 +313,7 @@ def nvfp4_linear(a_codes, a_sf, g_a, w_codes, w_sf, segments, g_seg, workspace, 
 
 
 def nvfp4_linear_bf16(x, g_a, w_codes, w_sf, segments, g_seg, workspace, out=None, out_f32: bool = False,
-                      stream=None) -> torch.Tensor:
+                      stream=None, w_resident: bool = False) -> torch.Tensor:
     """Same layer fed with bf16 activations; quantization happens inside the call."""
     assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
     M, K = x.shape
@@ -318,7 +321,7 @@ def nvfp4_linear_bf16(x, g_a, w_codes, w_sf, segments, g_seg, workspace, out=Non
     pairs = seg_pairs(segments)
     if out is None:
         out = torch.empty((M, N), dtype=torch.float32 if out_f32 else torch.bfloat16, device=x.device)
-    flags = (OUT_F32 if out.dtype == torch.float32 else OUT_BF16) | WS_ZEROED
+    flags = (OUT_F32 if out.dtype == torch.float32 else OUT_BF16) | WS_ZEROED | (W_RESIDENT if w_resident else 0)
     _check(lib().nvfp4_linear_bf16(_ptr(x), x.stride(0), _ptr(g_a), M, K, _ptr(w_codes), _ptr(w_sf), N,
                                    _segments(pairs), _ptr(g_seg), len(pairs), _ptr(out), out.stride(0), flags,
                                    _ptr(workspace), workspace.numel(), _stream(stream)), "nvfp4_linear_bf16")

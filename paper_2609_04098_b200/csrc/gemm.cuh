@@ -52,6 +52,9 @@ struct GemmParams {
     int32_t k_tiles;         // ceil(K / 256)
     int32_t katoms;          // K / 64: 512-byte scale atoms per 128-row band
     int32_t group_m;         // row units per raster group (see tile_of)
+    int32_t a_box_bytes;     // bytes of one A code box: 128 rows x 128 bytes, fewer rows for decode-sized M
+                             // (the tensor core still multiplies 128 rows; what the rows past the box hold in
+                             // shared memory only reaches accumulator rows that are never stored)
     // split-K (small M): an output tile is computed by split_k CTAs, each over k_per_split
     // consecutive K tiles; partial sums meet in `partial` (fp32 [rows padded to 128][ldp], zero
     // between calls), `counters` (one per tile and lane quarter, zero between calls) tell the
@@ -74,7 +77,7 @@ struct GemmParams {
     void* dbg_y;             // optional testing outputs: bf16 [M, 2 * inner] (interleaved columns) ...
     void* dbg_h;             // ... and bf16 [M, inner]
 };
-constexpr int kEpiPlain = 0, kEpiSwiglu = 1;
+constexpr int kEpiPlain = 0, kEpiSwiglu = 1, kEpiClusterSplit = 2;
 
 constexpr int kGemmThreads = 224;
 constexpr int kBM = 128;
@@ -84,7 +87,11 @@ constexpr int kTmemCols = 512;
 constexpr int kOutPieceCols = 64;             // epilogue piece: 32 rows x 64 bf16 = 4 KB
 constexpr int kOutPieceBytes = 32 * kOutPieceCols * 2;
 
-template <int BN, int STAGES, bool PAIR>
+constexpr int kClusterSplitSlotBytes = 32 * 128 * 4;      // fp32 partial sums of one 32-row quarter of a 128-wide tile
+constexpr int kClusterSplitSlots = 5;                     // landing slots in the cluster's first CTA
+constexpr int kDefaultOutBytes = 4 * 2 * kOutPieceBytes;  // per epilogue warp: two pieces
+
+template <int BN, int STAGES, bool PAIR, int OUT_BYTES_ = kDefaultOutBytes>
 struct GemmCfg {
     // Two TMEM accumulators.  BN = 128: disjoint (0..127, 128..255).  BN = 256: they do not both
     // fit beside the scale columns, so they OVERLAP by one epilogue piece: columns 0..255 and
@@ -102,7 +109,7 @@ struct GemmCfg {
     static constexpr int SFA_BYTES = kStepsPerStage * 512;
     static constexpr int SFB_BYTES = NB_BANDS * kStepsPerStage * 512;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;
-    static constexpr int OUT_BYTES = 4 * 2 * kOutPieceBytes;           // per epilogue warp: two pieces
+    static constexpr int OUT_BYTES = OUT_BYTES_;                       // output staging (or the cluster split's landing slots)
     static constexpr int BAR_BYTES = (2 * STAGES + 2 * ACC + 1) * 8 + 16;
     static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + OUT_BYTES + BAR_BYTES;
     // TMEM columns: accumulators first, then the scale columns (one set per smem stage, or a
@@ -129,12 +136,19 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 // EPI: kEpiPlain writes Y; kEpiSwiglu (BN = 256 only) turns every 32 accumulator columns -- 16 gate
 // and 16 up values of one row -- into one 16-element block of h = bf16(silu(bf16(gate)) * bf16(up))
 // and writes its NVFP4 codes and scale byte: the 4 bytes per element that Y would cost become 0.5625.
+// kEpiClusterSplit (decode-sized M, BN = 128, K a multiple of 256): the `split_k` CTAs of a cluster share
+// ONE output tile along K -- CTA r runs K tiles [r, r + 1) * k_per_split -- so that a layer with fewer
+// tiles than SMs still pulls its weights through every SM's load path and spreads the MMA issue work.
+// CTAs 1.. push their fp32 partial sums into landing slots in CTA 0's shared memory with bulk copies
+// that count their bytes on a barrier of CTA 0; CTA 0 waits for that barrier, adds the
+// slots to its own accumulator in a fixed order, applies the scales and writes Y.  One tile per
+// cluster; nothing goes through global memory, nothing has to be zeroed, and no fence is needed.
 template <int BN, int STAGES, bool PAIR, bool FULLK, int EPI = kEpiPlain>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const __grid_constant__ CUtensorMap tmSFA, const __grid_constant__ CUtensorMap tmSFB,
             const __grid_constant__ CUtensorMap tmY, const __grid_constant__ GemmParams p) {
-    using C = GemmCfg<BN, STAGES, PAIR>;
+    using C = GemmCfg<BN, STAGES, PAIR, EPI == kEpiClusterSplit ? kClusterSplitSlots * kClusterSplitSlotBytes : kDefaultOutBytes>;
     constexpr int ACC = C::ACC;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -147,17 +161,25 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     uint64_t* drain = tempty + ACC;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 1);
     volatile uint32_t* abort_flag = tmem_slot + 1;
+    uint64_t* cs_ready = reinterpret_cast<uint64_t*>(tmem_slot + 2);   // cluster split: the other CTAs' partial sums are in place
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const uint32_t rank = PAIR ? ptx::cluster_ctarank() : 0u;          // 0 = leader
-    const uint32_t unit_id = PAIR ? (blockIdx.x >> 1) : blockIdx.x;    // CTA or cluster index
-    const uint32_t n_units = PAIR ? (gridDim.x >> 1) : gridDim.x;
+    constexpr bool CSPLIT = EPI == kEpiClusterSplit;
+    static_assert(!CSPLIT || (BN == 128 && !PAIR && FULLK), "cluster split-K: 128 x 128 tiles, whole K tiles");
+    const uint32_t csize = CSPLIT ? static_cast<uint32_t>(p.split_k) : 1u;    // CTAs that share a tile along K
+    const uint32_t crank = CSPLIT ? ptx::cluster_ctarank() : 0u;              // which part of K is this CTA's
+    const uint32_t unit_id = PAIR ? (blockIdx.x >> 1) : (CSPLIT ? blockIdx.x / csize : blockIdx.x);    // CTA or cluster index
+    const uint32_t n_units = PAIR ? (gridDim.x >> 1) : (CSPLIT ? gridDim.x / csize : gridDim.x);
     const uint32_t m_units = PAIR ? (static_cast<uint32_t>(p.m_tiles) + 1u) >> 1 : static_cast<uint32_t>(p.m_tiles);
-    const uint32_t split_k = static_cast<uint32_t>(p.split_k);
+    const uint32_t split_k = CSPLIT ? 1u : static_cast<uint32_t>(p.split_k);
     const uint32_t total_tiles = m_units * static_cast<uint32_t>(p.n_tiles) * split_k;    // work items
     const uint32_t my_tiles = total_tiles > unit_id ? (total_tiles - unit_id + n_units - 1) / n_units : 0u;
-    const uint32_t k_tiles = static_cast<uint32_t>(p.k_per_split);                        // K tiles per item
+    const int32_t cs_kt0 = static_cast<int32_t>(crank) * p.k_per_split;       // cluster split: this CTA's K tiles
+    const int32_t cs_kt1 = min(cs_kt0 + p.k_per_split, p.k_tiles);
+    const uint32_t k_tiles = CSPLIT ? static_cast<uint32_t>(cs_kt1 - cs_kt0)
+                                    : static_cast<uint32_t>(p.k_per_split);              // K tiles per item
     const uint32_t total_it = my_tiles * k_tiles;
     const uint32_t peer_abort =
         PAIR ? ptx::mapa_shared(ptx::smem_u32(const_cast<uint32_t*>(abort_flag)), rank ^ 1u) : 0u;
@@ -172,6 +194,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             ptx::mbar_init(&tempty[a], 4 * C::CTAS);     // epilogue warps of every CTA of the tile
         }
         ptx::mbar_init(drain, 1);
+        if (CSPLIT) {
+            // completes when every other CTA's partial sums (its live 32-row quarters, all 128 columns) have landed
+            const uint32_t live_q = static_cast<uint32_t>(min(p.M, kBM) + 31) >> 5;
+            ptx::mbar_init(cs_ready, 1);
+            if (crank == 0u) ptx::mbar_arrive_expect_tx(cs_ready, (csize - 1u) * live_q * kClusterSplitSlotBytes);
+        }
         *abort_flag = 0u;
         ptx::fence_barrier_init();
     }
@@ -180,7 +208,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         else      { ptx::tmem_alloc(tmem_slot, kTmemCols);      ptx::tmem_relinquish(); }
     }
     ptx::tc_fence_before();
-    if (PAIR) ptx::cluster_sync_all(); else __syncthreads();   // barriers and TMEM exist from here on
+    // barriers and TMEM exist from here on (cluster split: the barrier-init fence above is what makes
+    // CTA 0's barrier visible to the other CTAs' remote copies; the cluster barrier only has to order execution)
+    if (PAIR) ptx::cluster_sync_all(); else if (CSPLIT) ptx::cluster_sync_relaxed(); else __syncthreads();
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     // CTA 0 leaves its own clock readings in the status block (words 2..9: cycle counter and wall clock
@@ -190,10 +220,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         reinterpret_cast<unsigned long long*>(p.status)[1] = static_cast<unsigned long long>(clock64());
         reinterpret_cast<unsigned long long*>(p.status)[2] = ptx::globaltimer_ns();
     }
-    // Everything above ran while the kernel in front of this one (the activation quantizer, which
-    // releases its dependents early) may still have been working; nothing below may read global
-    // memory before that kernel has finished.
-    ptx::pdl_wait();
+    // This kernel may have been started while the kernel in front of it (the activation quantizer or
+    // another GEMM, which release their dependents early) was still working, and it releases its own
+    // dependents right away: they all wait (pdl_wait) before they touch anything a predecessor may
+    // still read or write.  Here every role waits at its first access to such memory: the A producer
+    // before its first load, the epilogue before it reads the global scales or writes Y, the W producer
+    // too -- unless the caller has said that the weights were complete long before (NVFP4_W_RESIDENT):
+    // then the weight stream of this layer starts under the tail of the previous one.
+    ptx::pdl_launch_dependents();
 
     // tile index -> (row unit, column tile).  Tiles are visited in groups of `group_m` row
     // units; inside a group the row unit varies fastest, then the column tile.  The CTAs that
@@ -223,7 +257,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             ptx::prefetch_tensormap(tm_sf);
             const uint32_t code_off = is_a ? 0u : C::A_BYTES;
             const uint32_t sf_off = C::A_BYTES + C::B_BYTES + (is_a ? 0u : C::SFA_BYTES);
-            const uint32_t tx = is_a ? (C::A_BYTES + C::SFA_BYTES) : (C::B_BYTES + C::SFB_BYTES);
+            const uint32_t tx = is_a ? (static_cast<uint32_t>(p.a_box_bytes) + C::SFA_BYTES) : (C::B_BYTES + C::SFB_BYTES);
+            if (is_a || (p.flags & NVFP4_W_RESIDENT) == 0u) ptx::pdl_wait();
             uint32_t it = 0;
             bool ok = true;
             for (uint32_t t = 0; ok && t < my_tiles; ++t) {
@@ -232,8 +267,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 const int32_t a_band = PAIR ? 2 * um + static_cast<int32_t>(rank) : um;
                 const int32_t code_row = is_a ? a_band * kBM : un * BN + static_cast<int32_t>(rank) * C::B_ROWS;
                 const int32_t sf_band = is_a ? a_band : un * C::NB_BANDS;
-                const int32_t kt_end = (ks + 1) * p.k_per_split;        // K tiles past the tensor load zeros
-                for (int32_t kt = ks * p.k_per_split; kt < kt_end; ++kt, ++it) {
+                const int32_t kt_end = CSPLIT ? cs_kt1 : (ks + 1) * p.k_per_split;    // K tiles past the tensor load zeros
+                for (int32_t kt = CSPLIT ? cs_kt0 : ks * p.k_per_split; kt < kt_end; ++kt, ++it) {
                     const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
                     if (!ptx::mbar_wait_bounded(&empty[s], ph ^ 1u, abort_flag, p.wait_limit_ns, peer_abort)) { ok = false; break; }
                     uint8_t* st = smem + s * C::STAGE_BYTES;
@@ -365,6 +400,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         // ------------------------------------------------------------ epilogue
         const int quarter = warp;                       // TMEM lanes this warp may read
         uint8_t* out_w = out_s + quarter * (2 * kOutPieceBytes);
+        ptx::pdl_wait();                                // the scales may come from, and Y may still be read by, a predecessor
         const float g_a = __ldg(p.g_a);
         const bool out_f32 = (p.flags & NVFP4_OUT_F32) != 0u;
         const bool use_tma = p.tma_store != 0u;
@@ -398,6 +434,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 }
                 areg[i] = a;
             }
+            // the scales are in registers BEFORE the wait below (otherwise the compiler sinks their loads to
+            // the first use, and a global-memory latency lands between "accumulator full" and the first store)
+#pragma unroll
+            for (int i = 0; i < BN / 32; ++i) asm volatile("" : "+f"(areg[i]));
             // one lane polls (try_wait suspends the thread in hardware between looks): 128 threads
             // spinning on the barrier would take shared-memory cycles away from the MMAs
             bool ok = true;
@@ -475,6 +515,123 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 }
                 continue;
             }
+            // one lane writes 64 finished values of its row (16-byte stores where the row allows them)
+            auto store_row_piece = [&](const float (&v)[64], int32_t row, int32_t col0) {
+                const bool vec_ok = (reinterpret_cast<uintptr_t>(p.y) & 15u) == 0 && (p.ldy & (out_f32 ? 3 : 7)) == 0 &&
+                                    col0 + kOutPieceCols <= p.N;
+                if (out_f32) {
+                    float* yr = reinterpret_cast<float*>(p.y) + static_cast<int64_t>(row) * p.ldy + col0;
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        if (vec_ok) {
+                            *reinterpret_cast<float4*>(yr + 4 * j) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 4; ++e)
+                                if (col0 + 4 * j + e < p.N) yr[4 * j + e] = v[4 * j + e];
+                        }
+                    }
+                } else {
+                    __nv_bfloat16* yr = reinterpret_cast<__nv_bfloat16*>(p.y) + static_cast<int64_t>(row) * p.ldy + col0;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        if (vec_ok) {
+                            *reinterpret_cast<uint4*>(yr + 8 * j) =
+                                make_uint4(pack_bf16x2(v[8 * j], v[8 * j + 1]), pack_bf16x2(v[8 * j + 2], v[8 * j + 3]),
+                                           pack_bf16x2(v[8 * j + 4], v[8 * j + 5]), pack_bf16x2(v[8 * j + 6], v[8 * j + 7]));
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 8; ++e)
+                                if (col0 + 8 * j + e < p.N) yr[8 * j + e] = __float2bfloat16_rn(v[8 * j + e]);
+                        }
+                    }
+                }
+            };
+            if (CSPLIT) {
+                // ---- cluster split-K.  Slot (c - 1) * live_q + quarter of CTA 0 holds CTA c's partial sums of
+                // that quarter as float4 cells [column / 4][lane]: written and read 16 bytes per lane, no bank conflicts.
+                const int32_t row = row0 + lane;
+                const bool quarter_live = row0 < p.M;              // warp-uniform: rows past M are never sent or stored
+                const uint32_t live_q = static_cast<uint32_t>(min(p.M, kBM) + 31) >> 5;
+                const uint32_t cell0 = ptx::smem_u32(out_s) + static_cast<uint32_t>(lane * 16);
+                if (crank != 0u) {
+                    if (quarter_live) {
+                        // registers -> this CTA's own stage buffers (idle: its K loop is over) -> one bulk copy
+                        // per quarter into the slot, which counts its bytes on CTA 0's barrier
+                        const uint32_t slot = (crank - 1u) * live_q + static_cast<uint32_t>(quarter);
+                        const uint32_t local = ptx::smem_u32(smem) + static_cast<uint32_t>(quarter) * kClusterSplitSlotBytes;
+#pragma unroll 1
+                        for (int pc = 0; pc < NP; ++pc) {
+                            uint32_t r[64];
+                            __syncwarp();
+                            ptx::tmem_ld_32x64(t_row + pc * kOutPieceCols, r);
+                            ptx::tmem_ld_wait();
+#pragma unroll
+                            for (int j = 0; j < 16; ++j)
+                                ptx::st_shared_v4(local + static_cast<uint32_t>((pc * 16 + j) * 512 + lane * 16), r[4 * j],
+                                                  r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+                        }
+                        ptx::fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0)
+                            ptx::bulk_copy_to_cluster(ptx::mapa_shared(ptx::smem_u32(out_s) + slot * kClusterSplitSlotBytes, 0u), local,
+                                                      kClusterSplitSlotBytes, ptx::mapa_shared(ptx::smem_u32(cs_ready), 0u));
+                    }
+                    continue;
+                }
+                if (lane == 0) ok = ptx::mbar_wait_bounded(cs_ready, 0u, abort_flag, p.wait_limit_ns, 0u);
+                ok = __shfl_sync(0xffffffffu, static_cast<int>(ok), 0) != 0;
+                if (!ok) break;
+                if (!quarter_live) continue;
+#pragma unroll 1
+                for (int pc = 0; pc < NP; ++pc) {
+                    const int32_t col0 = n0 + pc * kOutPieceCols;
+                    if (col0 >= p.N) break;
+                    uint32_t r[64];
+                    float v[64];
+                    __syncwarp();
+                    ptx::tmem_ld_32x64(t_row + pc * kOutPieceCols, r);
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 64; ++j) v[j] = __uint_as_float(r[j]);
+                    for (uint32_t c = 1; c < csize; ++c) {         // fixed order: the sum does not depend on timing
+                        const uint32_t cell = cell0 + ((c - 1u) * live_q + static_cast<uint32_t>(quarter)) * kClusterSplitSlotBytes +
+                                              static_cast<uint32_t>(pc * 16 * 512);
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const uint4 q = ptx::ld_shared_v4(cell + static_cast<uint32_t>(j * 512));
+                            v[4 * j] = __fadd_rn(v[4 * j], __uint_as_float(q.x));
+                            v[4 * j + 1] = __fadd_rn(v[4 * j + 1], __uint_as_float(q.y));
+                            v[4 * j + 2] = __fadd_rn(v[4 * j + 2], __uint_as_float(q.z));
+                            v[4 * j + 3] = __fadd_rn(v[4 * j + 3], __uint_as_float(q.w));
+                        }
+                    }
+#pragma unroll
+                    for (int j = 0; j < 64; ++j)
+                        v[j] = __fmul_rn(v[j], __shfl_sync(0xffffffffu, areg[pc * 2 + (j >> 5)], j & 31));
+                    if (use_tma) {
+                        // this piece's part of the first landing slot of this quarter is in registers by now:
+                        // it serves as the staging buffer of the TMA store (rows past M are clipped there)
+                        uint8_t* buf = out_s + quarter * kClusterSplitSlotBytes + pc * (kClusterSplitSlotBytes / NP);
+                        __syncwarp();
+                        const uint32_t row_s = ptx::smem_u32(buf) + lane * 128;
+#pragma unroll
+                        for (int c = 0; c < 8; ++c)     // 128-byte swizzle: 16-byte chunk index XOR (row mod 8)
+                            ptx::st_shared_v4(row_s + ((c ^ (lane & 7)) << 4), pack_bf16x2(v[8 * c + 0], v[8 * c + 1]),
+                                              pack_bf16x2(v[8 * c + 2], v[8 * c + 3]), pack_bf16x2(v[8 * c + 4], v[8 * c + 5]),
+                                              pack_bf16x2(v[8 * c + 6], v[8 * c + 7]));
+                        ptx::fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) {
+                            ptx::tma_store_2d(&tmY, buf, col0, row0);
+                            ptx::bulk_commit_group();
+                        }
+                    } else if (row < p.M) {
+                        store_row_piece(v, row, col0);
+                    }
+                }
+                continue;
+            }
             if (split_k > 1u) {
                 // ---- split-K: add this item's partial sums to the tile's fp32 buffer; the last of
                 // the split_k arrivals (per lane quarter) finishes the tile
@@ -529,35 +686,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     for (int j = 0; j < 64; ++j)
                         v[j] = __fmul_rn(v[j], __shfl_sync(0xffffffffu, areg[pc * 2 + (j >> 5)], j & 31));
                     if (!row_ok) continue;
-                    const bool vec_ok = (reinterpret_cast<uintptr_t>(p.y) & 15u) == 0 && (p.ldy & (out_f32 ? 3 : 7)) == 0 &&
-                                        col0 + kOutPieceCols <= p.N;
-                    if (out_f32) {
-                        float* yr = reinterpret_cast<float*>(p.y) + static_cast<int64_t>(row) * p.ldy + col0;
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            if (vec_ok) {
-                                *reinterpret_cast<float4*>(yr + 4 * j) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-                            } else {
-#pragma unroll
-                                for (int e = 0; e < 4; ++e)
-                                    if (col0 + 4 * j + e < p.N) yr[4 * j + e] = v[4 * j + e];
-                            }
-                        }
-                    } else {
-                        __nv_bfloat16* yr = reinterpret_cast<__nv_bfloat16*>(p.y) + static_cast<int64_t>(row) * p.ldy + col0;
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            if (vec_ok) {
-                                *reinterpret_cast<uint4*>(yr + 8 * j) =
-                                    make_uint4(pack_bf16x2(v[8 * j], v[8 * j + 1]), pack_bf16x2(v[8 * j + 2], v[8 * j + 3]),
-                                               pack_bf16x2(v[8 * j + 4], v[8 * j + 5]), pack_bf16x2(v[8 * j + 6], v[8 * j + 7]));
-                            } else {
-#pragma unroll
-                                for (int e = 0; e < 8; ++e)
-                                    if (col0 + 8 * j + e < p.N) yr[8 * j + e] = __float2bfloat16_rn(v[8 * j + e]);
-                            }
-                        }
-                    }
+                    store_row_piece(v, row, col0);
                 }
                 __syncwarp();
                 if (lane == 0) *counter = 0u;                      // ready for the next call
@@ -640,7 +769,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     // which signal this CTA's barriers): give them time to land before anything is torn down
     if (*abort_flag != 0u) __nanosleep(50000);
     ptx::tc_fence_before();
-    if (PAIR) ptx::cluster_sync_all(); else __syncthreads();   // nobody touches TMEM or a partner's barriers after this
+    // (cluster split: CTA 0 arrives here only after the copies into its shared memory have landed -- or,
+    // having given up, after the sleep above -- so the CTAs they read from are still alive while they run;
+    // no data passes through this barrier, so it carries no memory ordering)
+    if (PAIR) ptx::cluster_sync_all(); else if (CSPLIT) ptx::cluster_sync_relaxed(); else __syncthreads();   // nobody touches TMEM or a partner's barriers after this
     if (warp == 6) {
         ptx::tc_fence_after();
         if (PAIR) ptx::tmem_dealloc_pair(tmem_base, kTmemCols); else ptx::tmem_dealloc(tmem_base, kTmemCols);

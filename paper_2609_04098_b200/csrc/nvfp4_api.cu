@@ -1,6 +1,7 @@
 // Host side of the C ABI declared in include/nvfp4.h: argument checks, TMA
 // descriptor set-up (cached), tile-shape choice and launches.  No allocation,
 // no synchronisation (except nvfp4_device_status), nothing thrown.
+#include <array>
 #include <atomic>
 #include <cstdio>
 #include <cstdlib>
@@ -251,6 +252,74 @@ nvfp4_status launch_gemm(const GemmMaps& tm, GemmParams& p, int sm_count, cudaSt
     const int64_t use = tiles < units ? tiles : units;
     cfg.gridDim = dim3(static_cast<unsigned>((PAIR ? 2 : 1) * use), 1, 1);
     cudaError_t e = cudaLaunchKernelEx(&cfg, gemm_kernel<BN, STAGES, PAIR, FULLK, EPI>, tm.a, tm.b, tm.sfa, tm.sfb, tm.y, p);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return e == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+}
+
+// Decode-sized M with fewer 128 x 128 tiles than SMs: clusters of `S` CTAs share a tile along K and
+// meet in the shared memory of the cluster's first CTA (gemm.cuh, kEpiClusterSplit).  Picks the
+// largest S (2..6) for which every tile's cluster is resident at once, every CTA gets at least two
+// K tiles and the partial sums fit the landing slots, and launches; returns NVFP4_ERR_SHAPE without
+// launching when no such S exists.
+nvfp4_status launch_gemm_cluster_split(const GemmMaps& tm, GemmParams& p, int sm_count, cudaStream_t stream) {
+    constexpr int BN = 128, STAGES = 4, kMaxS = 1 + kClusterSplitSlots;
+    using C = GemmCfg<BN, STAGES, false, kClusterSplitSlots * kClusterSplitSlotBytes>;
+    auto kernel = gemm_kernel<BN, STAGES, false, true, kEpiClusterSplit>;
+    static std::mutex mu;
+    static std::unordered_map<int, std::array<int, kMaxS + 1>> resident;    // per device and S: clusters resident at once (0 = unset)
+    int dev = 0;
+    cudaGetDevice(&dev);
+    p.n_tiles = (p.N + BN - 1) / BN;
+    const int64_t tiles = static_cast<int64_t>(p.m_tiles) * p.n_tiles;
+    if (tiles <= 0 || tiles * 2 > sm_count || p.m_tiles != 1) return NVFP4_ERR_SHAPE;
+    p.group_m = p.m_tiles;
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof(cfg));
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.blockDim = dim3(kGemmThreads, 1, 1);
+    cfg.dynamicSmemBytes = C::SMEM_BYTES;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    int S = static_cast<int>(sm_count / tiles);
+    const int live_q = ((p.M < kBM ? p.M : kBM) + 31) / 32;      // 32-row quarters of the tile that hold rows of Y
+    if (S > 1 + kClusterSplitSlots / live_q) S = 1 + kClusterSplitSlots / live_q;
+    if (S > p.k_tiles / 2) S = p.k_tiles / 2;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        auto& r = resident[dev];
+        if (r[0] == 0) {
+            if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
+                return NVFP4_ERR_CUDA;
+            r[0] = 1;
+        }
+        for (; S >= 2; --S) {
+            if (r[S] == 0) {
+                attr[0].val.clusterDim.x = static_cast<unsigned>(S);
+                cfg.gridDim = dim3(static_cast<unsigned>(sm_count / S * S), 1, 1);
+                int n = 0;
+                if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
+                r[S] = n > 0 ? n : -1;
+            }
+            if (r[S] >= tiles) break;
+        }
+    }
+    if (S < 2) return NVFP4_ERR_SHAPE;
+    p.k_per_split = (p.k_tiles + S - 1) / S;
+    while (S > 2 && static_cast<int64_t>(S - 1) * p.k_per_split >= p.k_tiles) --S;     // every CTA has work
+    if (static_cast<int64_t>(S - 1) * p.k_per_split >= p.k_tiles) return NVFP4_ERR_SHAPE;
+    p.split_k = S;
+    p.partial = nullptr;
+    p.counters = nullptr;
+    attr[0].val.clusterDim.x = static_cast<unsigned>(S);
+    cfg.gridDim = dim3(static_cast<unsigned>(tiles * S), 1, 1);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, tm.a, tm.b, tm.sfa, tm.sfb, tm.y, p);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return e == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
@@ -648,7 +717,7 @@ nvfp4_status linear_impl(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const 
         return NVFP4_ERR_ALIGN;
     if (d_workspace == nullptr || workspace_bytes < kStatusBytes) return NVFP4_ERR_WORKSPACE;
     if (!aligned16(d_workspace)) return NVFP4_ERR_ALIGN;
-    if ((flags & ~(NVFP4_OUT_F32 | NVFP4_WS_ZEROED)) != 0u) return NVFP4_ERR_SHAPE;
+    if ((flags & ~(NVFP4_OUT_F32 | NVFP4_WS_ZEROED | NVFP4_W_RESIDENT)) != 0u) return NVFP4_ERR_SHAPE;
     if (M == 0 || N == 0) return NVFP4_OK;
     DeviceInfo info;
     st = check_arch(info);
@@ -661,7 +730,11 @@ nvfp4_status linear_impl(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const 
     std::memset(&tm, 0, sizeof(tm));
     // rows the code buffer really has (>= M): with whole 128-row boxes in bounds TMA takes no
     // out-of-bounds path, which is measurably slower; rows past M hold zero scales and are never stored
-    st = codes_tensor_map(d_a_codes, a_rows_alloc > M ? a_rows_alloc : M, K, kBM, &tm.a);
+    // Decode-sized M: the A box holds only the rows that exist (rounded up to the 8-row swizzle period).
+    // Every CTA reads the same A from L2 at the same moment; a full 128-row box there costs as much
+    // load-path time per stage as the W tile it is multiplied with.
+    const int a_box_rows = M < kBM ? static_cast<int>((M + 7) / 8 * 8) : kBM;
+    st = codes_tensor_map(d_a_codes, a_rows_alloc > M ? a_rows_alloc : M, K, a_box_rows, &tm.a);
     if (st != NVFP4_OK) return st;
     st = codes_tensor_map(d_w_codes, N, K, bn == 2 ? 128 : tile_n, &tm.b);
     if (st != NVFP4_OK) return st;
@@ -688,6 +761,7 @@ nvfp4_status linear_impl(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const 
     p.m_tiles = static_cast<int32_t>((M + kBM - 1) / kBM);
     p.k_tiles = static_cast<int32_t>((K + 255) / 256);
     p.katoms = static_cast<int32_t>(K / 64);
+    p.a_box_bytes = a_box_rows * kBKBytes;
     p.split_k = 1;
     p.k_per_split = p.k_tiles;
     if (bn == 128 && (flags & NVFP4_WS_ZEROED) != 0u && d_split != nullptr && (K % 256) == 0) {
@@ -728,6 +802,12 @@ nvfp4_status linear_impl(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const 
                                   : launch_gemm<256, 5, true, false, kEpiSwiglu>(tm, p, info.sm_count, s);
         return fullk ? launch_gemm<256, 3, false, true, kEpiSwiglu>(tm, p, info.sm_count, s)
                      : launch_gemm<256, 3, false, false, kEpiSwiglu>(tm, p, info.sm_count, s);
+    }
+    if (bn == 128 && fullk && M <= 128 && g_variant.load(std::memory_order_relaxed) == 0) {
+        // decode-sized and fewer tiles than half the machine: share each tile along K inside a cluster
+        GemmParams pc = p;
+        const nvfp4_status cst = launch_gemm_cluster_split(tm, pc, info.sm_count, s);
+        if (cst != NVFP4_ERR_SHAPE) return cst;
     }
     switch (bn) {
         case 128: return fullk ? launch_gemm<128, 5, false, true>(tm, p, info.sm_count, s) : launch_gemm<128, 5, false, false>(tm, p, info.sm_count, s);
@@ -786,7 +866,7 @@ nvfp4_status linear_bf16_impl(const void* d_x, int64_t ldx, const float* d_g_a, 
         d_y == nullptr)
         return NVFP4_ERR_NULL;
     if (ldx < K || ldy < N || M >= (1ll << 31) - 256 || N >= (1ll << 31) - 256 || K >= (1ll << 31)) return NVFP4_ERR_SHAPE;
-    if ((flags & ~(NVFP4_OUT_F32 | NVFP4_WS_ZEROED)) != 0u) return NVFP4_ERR_SHAPE;
+    if ((flags & ~(NVFP4_OUT_F32 | NVFP4_WS_ZEROED | NVFP4_W_RESIDENT)) != 0u) return NVFP4_ERR_SHAPE;
     nvfp4_status st = check_segments(segs, nseg, N);
     if (N == 0 && segs != nullptr) st = NVFP4_OK;
     if (st != NVFP4_OK) return st;

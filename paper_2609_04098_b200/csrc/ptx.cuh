@@ -127,6 +127,18 @@ __device__ __forceinline__ uint32_t cluster_ctarank() {
 __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+// execution barrier only: every thread of the cluster has arrived, no memory ordering implied
+__device__ __forceinline__ void cluster_sync_relaxed() {
+    asm volatile("barrier.cluster.arrive.relaxed.aligned;\n\tbarrier.cluster.wait.aligned;" ::: "memory");
+}
+// `bytes` (a multiple of 16) from this CTA's shared memory to another CTA's, asynchronously; their arrival
+// counts on that CTA's barrier `cluster_bar`, and a thread that sees the barrier's phase complete sees the data
+__device__ __forceinline__ void bulk_copy_to_cluster(uint32_t cluster_dst, uint32_t local_src, uint32_t bytes,
+                                                     uint32_t cluster_bar) {
+    asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(cluster_dst), "r"(local_src), "r"(bytes), "r"(cluster_bar)
+                 : "memory");
+}
 // address of the same shared-memory variable in CTA `rank` of this cluster
 __device__ __forceinline__ uint32_t mapa_shared(uint32_t local_saddr, uint32_t rank) {
     uint32_t r;

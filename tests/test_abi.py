@@ -73,7 +73,7 @@ def test_host_side_argument_checks_need_no_gpu(L):
     assert lin(ws=None) == 5
     assert lin(wsb=8) == 5
     assert lin(a=vp(0x1004)) == 3
-    assert lin(flags=6) == 2
+    assert lin(flags=8) == 2 and lin(flags=14) == 2
     assert L.nvfp4_workspace_reset(None, 256, None) == 1
     assert L.nvfp4_workspace_reset(p, 8, None) == 5
     assert L.nvfp4_device_status(None, None) == 1
@@ -90,7 +90,7 @@ def test_host_side_argument_checks_need_no_gpu(L):
     assert fused(K=48) == 2
     assert fused(ldx=32) == 2
     assert fused(ldy=8) == 2
-    assert fused(flags=4) == 2
+    assert fused(flags=8) == 2
     assert fused(N=24, ldy=32) == 4
     assert fused(ws=None) == 5
     assert fused(wsb=4096) == 5

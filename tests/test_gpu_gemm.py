@@ -34,13 +34,13 @@ def _oracle_operands(seed, M, K, segspec, hot=2):
     return segs, x, w, ac, asf, ga, wc, wsf, gs
 
 
-def _run_from_oracle_operands(segs, ac, asf, ga, wc, wsf, gs, K, out_f32=False, ws=None):
+def _run_from_oracle_operands(segs, ac, asf, ga, wc, wsf, gs, K, out_f32=False, ws=None, w_resident=False):
     """Feed the ORACLE's codes and scales (re-ordered by the oracle's own layout map) to
     the GPU GEMM: a layout disagreement with the hardware shows up as a wrong product."""
     ws = ws if ws is not None else _ws()
     y = nv.nvfp4_linear(gu.dev_u8(ac), gu.dev_u8(oracle.sf_to_mma(asf, K)), gu.dev_f32(ga),
                         gu.dev_u8(wc), gu.dev_u8(oracle.sf_to_mma(wsf, K)), segs, gu.dev_f32(gs), ws,
-                        out_f32=out_f32)
+                        out_f32=out_f32, w_resident=w_resident)
     assert nv.device_status(ws) == 0
     return y
 
@@ -204,10 +204,15 @@ def test_gdn_in_projection_full_size_sampled(variant):
     _check_sampled(y, M, N, K, segs, ac, asf, ga, wc, wsf, gcol, np.random.default_rng(0), "gdn")
 
 
-# ---- decode-sized batches: split-K over a self-cleaning workspace -----------------------------
-@pytest.mark.parametrize("M,N,K", [(1, 6144, 5120), (16, 520, 8192), (100, 2064, 8448), (128, 1000, 9216), (3, 136, 17408)])
+# ---- decode-sized batches: K shared by the CTAs of a cluster, or split over a self-cleaning workspace ----
+# automatic choice: clusters whose CTAs meet in shared memory (every shape below has few enough tiles);
+# variant 128 forced: one CTA per tile, K split through the workspace where K is long enough
+@pytest.mark.parametrize("M,N,K", [(1, 6144, 5120), (16, 520, 8192), (33, 1100, 5120), (64, 6144, 5120), (100, 2064, 8448),
+                                   (128, 1000, 9216), (3, 136, 17408), (7, 128, 512)])
 @pytest.mark.parametrize("out_f32", [False, True])
-def test_small_m_split_k(M, N, K, out_f32):
+@pytest.mark.parametrize("variant", [0, 128])
+def test_small_m_split_k(M, N, K, out_f32, variant):
+    nv.set_gemm_variant(variant)
     n1 = N // 3
     segs, x, w, ac, asf, ga, wc, wsf, gs = _oracle_operands(17, M, K, (("p", n1, 0.02), ("q", N - n1, 0.2)))
     gcol = oracle.col_scales(N, segs, gs)
@@ -216,17 +221,21 @@ def test_small_m_split_k(M, N, K, out_f32):
     ws = nv.alloc_workspace(gu.DEV, M, N, K, 2)            # zero-filled, large enough for the split-K area
     assert ws.numel() > 256
     first = None
-    for _ in range(3):                                      # the same workspace every time: it must come back clean
-        y = _run_from_oracle_operands(segs, ac, asf, ga, wc, wsf, gs, K, out_f32=out_f32, ws=ws)
+    for rep in range(3):                                    # the same workspace every time: it must come back clean
+        y = _run_from_oracle_operands(segs, ac, asf, ga, wc, wsf, gs, K, out_f32=out_f32, ws=ws, w_resident=rep == 2)
         gu.check_gemm(y, y_ref, bound, "split-K %s" % ((M, N, K),))
         if first is None:
             first = y.clone()
+        elif variant == 0:
+            assert torch.equal(y, first)                    # the cluster adds its partial sums in a fixed order
         elif out_f32:
             # fp32 atomics add in arrival order: equal up to summation order
             assert torch.allclose(y, first, rtol=1e-5, atol=1e-6 * float(first.abs().max()))
     assert bool((ws[256:] == 0).all())                     # counters and partial sums left at zero
     # and the one-tile-per-CTA kernel gives the same answer (within summation order)
+    nv.set_gemm_variant(128)
     y1 = _run_from_oracle_operands(segs, ac, asf, ga, wc, wsf, gs, K, out_f32=out_f32)    # 256-byte workspace: no split
+    nv.set_gemm_variant(0)
     gu.check_gemm(y1, y_ref, bound, "no split")
 
 
