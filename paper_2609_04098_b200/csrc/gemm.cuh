@@ -76,6 +76,10 @@ struct GemmParams {
     int32_t inner;
     void* dbg_y;             // optional testing outputs: bf16 [M, 2 * inner] (interleaved columns) ...
     void* dbg_h;             // ... and bf16 [M, inner]
+    // activations quantized inside the kernel (EPI == kEpiClusterSplit only, a handful of rows): bf16
+    // [M, K] with row stride ldx; then no quantized copy of A exists in global memory at all
+    const uint16_t* x;
+    int64_t ldx;
 };
 constexpr int kEpiPlain = 0, kEpiSwiglu = 1, kEpiClusterSplit = 2;
 
@@ -143,6 +147,10 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 // that count their bytes on a barrier of CTA 0; CTA 0 waits for that barrier, adds the
 // slots to its own accumulator in a fixed order, applies the scales and writes Y.  One tile per
 // cluster; nothing goes through global memory, nothing has to be zeroed, and no fence is needed.
+// For a handful of rows the same variant also takes A as bf16 (GemmParams::x): the four epilogue warps
+// quantize each K tile of A straight into the stage buffer (codes in the 128-byte swizzle, scale bytes in
+// the atom layout, bit for bit what the quantize kernel would have written), which removes that kernel
+// and its launch from the chain; every CTA quantizes the K range it multiplies.
 template <int BN, int STAGES, bool PAIR, bool FULLK, int EPI = kEpiPlain>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
@@ -186,7 +194,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            ptx::mbar_init(&full[s], 2 * C::CTAS);       // the two producer threads of every CTA of the tile
+            // the two producer threads of every CTA of the tile; with A quantized in the kernel, the W
+            // producer and the four quantizing warps
+            ptx::mbar_init(&full[s], (CSPLIT && p.x != nullptr) ? 5 : 2 * C::CTAS);
             ptx::mbar_init(&empty[s], 1);
         }
         for (int a = 0; a < ACC; ++a) {
@@ -248,7 +258,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 
     if (warp == 4 || warp == 5) {
         // ------------------------------------------------------------ TMA producers
-        if (lane == 0) {
+        if (lane == 0 && !(CSPLIT && warp == 4 && p.x != nullptr)) {
             const bool is_a = warp == 4;
             const uint32_t leader_full = PAIR ? ptx::mapa_shared(ptx::smem_u32(full), 0u) : 0u;
             const CUtensorMap* tm_codes = is_a ? &tmA : &tmB;
@@ -414,6 +424,68 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 bad = bad || !(gs > 0.0f && gs <= 3.402823466e38f);
             }
             if (__any_sync(0xffffffffu, bad) && lane == 0) atomicExch(p.status, static_cast<uint32_t>(NVFP4_ERR_SCALE));
+        }
+        if (CSPLIT && p.x != nullptr && my_tiles != 0u) {
+            // ---- A from bf16.  Block b of a K tile = (row, 16-element block) with b = row * 16 + block; thread t
+            // takes blocks t, t + 128, ... (16 neighbouring threads read the 512 contiguous bytes of one row).
+            // The tile after the current one is loaded and quantized into registers while the stage it goes
+            // to is still being read by the tensor core; only the shared-memory stores wait for the stage.
+            constexpr int NB = 2;                                     // blocks per thread: up to 16 rows
+            const int nb = (p.a_box_bytes / kBKBytes) >> 3;           // ... of which this call uses rows / 8
+            const float c1 = __fdiv_rn(1.0f, __fmul_rn(6.0f, g_a));
+            const int32_t r0 = static_cast<int32_t>(threadIdx.x) >> 4, kb = static_cast<int32_t>(threadIdx.x) & 15;
+            uint4 lo[NB], hi[NB];
+            auto load_tile = [&](int32_t kt) {
+#pragma unroll
+                for (int b = 0; b < NB; ++b) {
+                    if (b >= nb) break;
+                    const int32_t r = r0 + 8 * b;
+                    lo[b] = make_uint4(0u, 0u, 0u, 0u);
+                    hi[b] = lo[b];
+                    if (r < p.M) {
+                        const uint4* src = reinterpret_cast<const uint4*>(p.x + static_cast<int64_t>(r) * p.ldx +
+                                                                          static_cast<int64_t>(kt) * 256 + kb * 16);
+                        lo[b] = __ldg(src);
+                        hi[b] = __ldg(src + 1);
+                    }
+                }
+            };
+            load_tile(cs_kt0);
+            bool ok = true;
+            uint32_t itq = 0;
+            for (int32_t kt = cs_kt0; ok && kt < cs_kt1; ++kt, ++itq) {
+                uint2 w[NB];
+                uint32_t s8[NB];
+#pragma unroll
+                for (int b = 0; b < NB; ++b) {
+                    if (b >= nb) break;
+                    const uint32_t hw[8] = {lo[b].x, lo[b].y, lo[b].z, lo[b].w, hi[b].x, hi[b].y, hi[b].z, hi[b].w};
+                    // rows past M: zero codes, zero scale (without the quantizer: its division takes the slow path on 1 / 0)
+                    w[b] = make_uint2(0u, 0u);
+                    s8[b] = 0u;
+                    if (r0 + 8 * b < p.M) w[b] = quantize_block(hw, g_a, c1, s8[b]);
+                }
+                if (kt + 1 < cs_kt1) load_tile(kt + 1);
+                const uint32_t s = itq % STAGES, ph = (itq / STAGES) & 1u;
+                if (lane == 0) ok = ptx::mbar_wait_bounded(&empty[s], ph ^ 1u, abort_flag, p.wait_limit_ns, 0u);
+                ok = __shfl_sync(0xffffffffu, static_cast<int>(ok), 0) != 0;
+                if (!ok) break;
+                const uint32_t st = ptx::smem_u32(smem) + s * C::STAGE_BYTES;
+#pragma unroll
+                for (int b = 0; b < NB; ++b) {
+                    const int32_t r = r0 + 8 * b;
+                    if (b < nb) {
+                        // 8 code bytes: 16-byte chunk (kb / 2) XOR (row mod 8) of the row's 128-byte swizzle line
+                        ptx::st_shared_v2(st + static_cast<uint32_t>(r * 128 + (((kb >> 1) ^ (r & 7)) << 4) + (kb & 1) * 8), w[b].x, w[b].y);
+                        // scale byte: atom kb / 4 of the stage, (row mod 32) * 16 + (row / 32) * 4 + kb mod 4
+                        ptx::st_shared_u8(st + static_cast<uint32_t>(C::A_BYTES + C::B_BYTES + (kb >> 2) * 512 + (r & 31) * 16 +
+                                                                     (r >> 5) * 4 + (kb & 3)), s8[b]);
+                    }
+                }
+                ptx::fence_proxy_async_smem();                        // the tensor core reads these bytes through the async proxy
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&full[s]);
+            }
         }
         uint32_t pieces_stored = 0;
         for (uint32_t t = 0; t < my_tiles; ++t) {

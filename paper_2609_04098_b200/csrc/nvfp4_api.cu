@@ -260,8 +260,10 @@ nvfp4_status launch_gemm(const GemmMaps& tm, GemmParams& p, int sm_count, cudaSt
 // meet in the shared memory of the cluster's first CTA (gemm.cuh, kEpiClusterSplit).  Picks the
 // largest S (2..6) for which every tile's cluster is resident at once, every CTA gets at least two
 // K tiles and the partial sums fit the landing slots, and launches; returns NVFP4_ERR_SHAPE without
-// launching when no such S exists.
-nvfp4_status launch_gemm_cluster_split(const GemmMaps& tm, GemmParams& p, int sm_count, cudaStream_t stream) {
+// launching when no such S exists -- unless `allow_single` (the caller wants this variant for its
+// in-kernel activation quantization): then S = 1, one CTA per tile, is the fallback.
+nvfp4_status launch_gemm_cluster_split(const GemmMaps& tm, GemmParams& p, int sm_count, cudaStream_t stream,
+                                       bool allow_single) {
     constexpr int BN = 128, STAGES = 4, kMaxS = 1 + kClusterSplitSlots;
     using C = GemmCfg<BN, STAGES, false, kClusterSplitSlots * kClusterSplitSlotBytes>;
     auto kernel = gemm_kernel<BN, STAGES, false, true, kEpiClusterSplit>;
@@ -271,7 +273,8 @@ nvfp4_status launch_gemm_cluster_split(const GemmMaps& tm, GemmParams& p, int sm
     cudaGetDevice(&dev);
     p.n_tiles = (p.N + BN - 1) / BN;
     const int64_t tiles = static_cast<int64_t>(p.m_tiles) * p.n_tiles;
-    if (tiles <= 0 || tiles * 2 > sm_count || p.m_tiles != 1) return NVFP4_ERR_SHAPE;
+    if (tiles <= 0 || p.m_tiles != 1) return NVFP4_ERR_SHAPE;
+    if (tiles * 2 > sm_count && !allow_single) return NVFP4_ERR_SHAPE;
     p.group_m = p.m_tiles;
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof(cfg));
@@ -310,10 +313,14 @@ nvfp4_status launch_gemm_cluster_split(const GemmMaps& tm, GemmParams& p, int sm
             if (r[S] >= tiles) break;
         }
     }
-    if (S < 2) return NVFP4_ERR_SHAPE;
+    if (S < 2 && !allow_single) return NVFP4_ERR_SHAPE;
+    if (S < 1) S = 1;
     p.k_per_split = (p.k_tiles + S - 1) / S;
-    while (S > 2 && static_cast<int64_t>(S - 1) * p.k_per_split >= p.k_tiles) --S;     // every CTA has work
-    if (static_cast<int64_t>(S - 1) * p.k_per_split >= p.k_tiles) return NVFP4_ERR_SHAPE;
+    while (S > 1 && static_cast<int64_t>(S - 1) * p.k_per_split >= p.k_tiles) {          // every CTA has work
+        --S;
+        p.k_per_split = (p.k_tiles + S - 1) / S;
+    }
+    if (S < 2 && !allow_single) return NVFP4_ERR_SHAPE;
     p.split_k = S;
     p.partial = nullptr;
     p.counters = nullptr;
@@ -704,8 +711,11 @@ nvfp4_status linear_impl(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const 
                          int64_t K, const uint8_t* d_w_codes, const uint8_t* d_w_sf, int64_t N,
                          const nvfp4_segment* segs, const float* d_g_seg, int nseg, void* d_y, int64_t ldy,
                          uint32_t flags, void* d_workspace, size_t workspace_bytes, void* d_split, size_t split_bytes,
-                         void* stream, int64_t a_rows_alloc = 0, const GemmParams* fused = nullptr) {
-    if (d_a_codes == nullptr || d_a_sf == nullptr || d_g_a == nullptr || d_w_codes == nullptr ||
+                         void* stream, int64_t a_rows_alloc = 0, const GemmParams* fused = nullptr,
+                         const uint16_t* aq_x = nullptr, int64_t aq_ldx = 0) {
+    // aq_x: bf16 activations that the kernel quantizes itself (the caller has checked that the shape
+    // takes the cluster-split variant); then there are no A codes or scales
+    if (((d_a_codes == nullptr || d_a_sf == nullptr) && aq_x == nullptr) || d_g_a == nullptr || d_w_codes == nullptr ||
         d_w_sf == nullptr || d_g_seg == nullptr || (d_y == nullptr && fused == nullptr))
         return NVFP4_ERR_NULL;
     if (M < 0 || N < 0 || K <= 0 || (K % 64) != 0 || ldy < N) return NVFP4_ERR_SHAPE;
@@ -713,7 +723,7 @@ nvfp4_status linear_impl(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const 
     nvfp4_status st = check_segments(segs, nseg, N);
     if (N == 0 && segs != nullptr) st = NVFP4_OK;
     if (st != NVFP4_OK) return st;
-    if (!aligned16(d_a_codes) || !aligned16(d_w_codes) || !aligned16(d_a_sf) || !aligned16(d_w_sf))
+    if ((aq_x == nullptr && (!aligned16(d_a_codes) || !aligned16(d_a_sf))) || !aligned16(d_w_codes) || !aligned16(d_w_sf))
         return NVFP4_ERR_ALIGN;
     if (d_workspace == nullptr || workspace_bytes < kStatusBytes) return NVFP4_ERR_WORKSPACE;
     if (!aligned16(d_workspace)) return NVFP4_ERR_ALIGN;
@@ -734,11 +744,11 @@ nvfp4_status linear_impl(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const 
     // Every CTA reads the same A from L2 at the same moment; a full 128-row box there costs as much
     // load-path time per stage as the W tile it is multiplied with.
     const int a_box_rows = M < kBM ? static_cast<int>((M + 7) / 8 * 8) : kBM;
-    st = codes_tensor_map(d_a_codes, a_rows_alloc > M ? a_rows_alloc : M, K, a_box_rows, &tm.a);
+    if (aq_x == nullptr) st = codes_tensor_map(d_a_codes, a_rows_alloc > M ? a_rows_alloc : M, K, a_box_rows, &tm.a);
     if (st != NVFP4_OK) return st;
     st = codes_tensor_map(d_w_codes, N, K, bn == 2 ? 128 : tile_n, &tm.b);
     if (st != NVFP4_OK) return st;
-    st = scales_tensor_map(d_a_sf, M, K, 1, &tm.sfa);
+    if (aq_x == nullptr) st = scales_tensor_map(d_a_sf, M, K, 1, &tm.sfa);
     if (st != NVFP4_OK) return st;
     st = scales_tensor_map(d_w_sf, N, K, tile_n / 128, &tm.sfb);
     if (st != NVFP4_OK) return st;
@@ -806,9 +816,12 @@ nvfp4_status linear_impl(const uint8_t* d_a_codes, const uint8_t* d_a_sf, const 
     if (bn == 128 && fullk && M <= 128 && g_variant.load(std::memory_order_relaxed) == 0) {
         // decode-sized and fewer tiles than half the machine: share each tile along K inside a cluster
         GemmParams pc = p;
-        const nvfp4_status cst = launch_gemm_cluster_split(tm, pc, info.sm_count, s);
-        if (cst != NVFP4_ERR_SHAPE) return cst;
+        pc.x = aq_x;
+        pc.ldx = aq_ldx;
+        const nvfp4_status cst = launch_gemm_cluster_split(tm, pc, info.sm_count, s, aq_x != nullptr);
+        if (cst != NVFP4_ERR_SHAPE || aq_x != nullptr) return cst;
     }
+    if (aq_x != nullptr) return NVFP4_ERR_SHAPE;
     switch (bn) {
         case 128: return fullk ? launch_gemm<128, 5, false, true>(tm, p, info.sm_count, s) : launch_gemm<128, 5, false, false>(tm, p, info.sm_count, s);
         case 256: return fullk ? launch_gemm<256, 3, false, true>(tm, p, info.sm_count, s) : launch_gemm<256, 3, false, false>(tm, p, info.sm_count, s);
@@ -854,6 +867,14 @@ size_t fused_min_bytes(int64_t M, int64_t K) {
     return kFusedCodesOffset + fused_codes_bytes(M, K) + sf;
 }
 
+// rows up to which nvfp4_linear_bf16 quantizes the activations inside the GEMM kernel: every CTA
+// quantizes the K range it multiplies, 48 times over for a 6144-wide layer.  The four warps that do
+// it are otherwise idle during the main loop, but each of them sits alone on its scheduler: one
+// 16-element block per thread and K tile (8 rows) hides under the weight stream (measured, 5120 ->
+// 6144, CUDA-graph replay: 9.5-10.0 us against 11.5 us with the quantize kernel in front), two
+// blocks per thread (9 to 16 rows) do not (11.0-11.9 us).
+constexpr int64_t kInKernelQuantRows = 8;
+
 // nvfp4_linear_bf16 on a workspace of the layout above; every argument is checked before
 // anything is enqueued
 nvfp4_status linear_bf16_impl(const void* d_x, int64_t ldx, const float* d_g_a, int64_t M, int64_t K,
@@ -876,9 +897,10 @@ nvfp4_status linear_bf16_impl(const void* d_x, int64_t ldx, const float* d_g_a, 
     const size_t min_bytes = fused_min_bytes(M, K);
     if (workspace_bytes < min_bytes) return NVFP4_ERR_WORKSPACE;
     if (M == 0 || N == 0) return NVFP4_OK;
-    // measured on B200 (5120 -> 6144, CUDA-graph replay): 1 / 2 tokens are faster through the
-    // weight-streaming kernel; from 3 tokens on the tensor cores win
-    if (M <= 2 && g_variant.load(std::memory_order_relaxed) == 0 && decode_smem_bytes(M, K) <= 200 * 1024) {
+    // measured on B200 (5120 -> 6144, CUDA-graph replay): one token is as fast through the
+    // weight-streaming kernel as through the tensor cores (9.7 us); two tokens take 12.7 us there and
+    // 9.7 us on the tensor cores, which need K to be a multiple of 256 to quantize A themselves
+    if (M <= (((K % 256) == 0) ? 1 : 2) && g_variant.load(std::memory_order_relaxed) == 0 && decode_smem_bytes(M, K) <= 200 * 1024) {
         // decode-sized batch: one weight-streaming kernel; of the workspace only the status word is used
         DeviceInfo info;
         st = check_arch(info);
@@ -905,6 +927,12 @@ nvfp4_status linear_bf16_impl(const void* d_x, int64_t ldx, const float* d_g_a, 
         return launch_decode<2>(dp, info.sm_count, s);
     }
     uint8_t* ws = reinterpret_cast<uint8_t*>(d_workspace);
+    if (M <= kInKernelQuantRows && (K % 256) == 0 && g_variant.load(std::memory_order_relaxed) == 0) {
+        // a handful of tokens: one kernel, which quantizes the K tiles of A it multiplies (gemm.cuh)
+        return linear_impl(nullptr, nullptr, d_g_a, M, K, d_w_codes, d_w_sf, N, segs, d_g_seg, nseg, d_y, ldy, flags,
+                           d_workspace, kStatusBytes, nullptr, 0, stream, 0, nullptr,
+                           reinterpret_cast<const uint16_t*>(d_x), ldx);
+    }
     uint8_t* codes = ws + kFusedCodesOffset;
     uint8_t* sf = codes + fused_codes_bytes(M, K);
     st = nvfp4_quantize_act(d_x, M, K, ldx, d_g_a, codes, sf, NVFP4_SF_MMA, stream);
