@@ -76,12 +76,12 @@ struct GemmParams {
     int32_t inner;
     void* dbg_y;             // optional testing outputs: bf16 [M, 2 * inner] (interleaved columns) ...
     void* dbg_h;             // ... and bf16 [M, inner]
-    // activations quantized inside the kernel (EPI == kEpiClusterSplit only, a handful of rows): bf16
+    // activations quantized inside the kernel (cluster-split builds only, a handful of rows): bf16
     // [M, K] with row stride ldx; then no quantized copy of A exists in global memory at all
     const uint16_t* x;
     int64_t ldx;
 };
-constexpr int kEpiPlain = 0, kEpiSwiglu = 1, kEpiClusterSplit = 2;
+constexpr int kEpiPlain = 0, kEpiSwiglu = 1, kEpiClusterSplit = 2, kEpiClusterSplitFew = 3;
 
 constexpr int kGemmThreads = 224;
 constexpr int kBM = 128;
@@ -92,7 +92,8 @@ constexpr int kOutPieceCols = 64;             // epilogue piece: 32 rows x 64 bf
 constexpr int kOutPieceBytes = 32 * kOutPieceCols * 2;
 
 constexpr int kClusterSplitSlotBytes = 32 * 128 * 4;      // fp32 partial sums of one 32-row quarter of a 128-wide tile
-constexpr int kClusterSplitSlots = 5;                     // landing slots in the cluster's first CTA
+// landing slots in the cluster's first CTA: five beside four stages, or two beside five stages
+__host__ __device__ constexpr int cluster_split_slots(int epi) { return epi == 2 ? 5 : (epi == 3 ? 2 : 0); }
 constexpr int kDefaultOutBytes = 4 * 2 * kOutPieceBytes;  // per epilogue warp: two pieces
 
 template <int BN, int STAGES, bool PAIR, int OUT_BYTES_ = kDefaultOutBytes>
@@ -140,7 +141,8 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 // EPI: kEpiPlain writes Y; kEpiSwiglu (BN = 256 only) turns every 32 accumulator columns -- 16 gate
 // and 16 up values of one row -- into one 16-element block of h = bf16(silu(bf16(gate)) * bf16(up))
 // and writes its NVFP4 codes and scale byte: the 4 bytes per element that Y would cost become 0.5625.
-// kEpiClusterSplit (decode-sized M, BN = 128, K a multiple of 256): the `split_k` CTAs of a cluster share
+// kEpiClusterSplit / kEpiClusterSplitFew (decode-sized M, BN = 128, K a multiple of 256; they differ only in how
+// shared memory is divided between stages and landing slots): the `split_k` CTAs of a cluster share
 // ONE output tile along K -- CTA r runs K tiles [r, r + 1) * k_per_split -- so that a layer with fewer
 // tiles than SMs still pulls its weights through every SM's load path and spreads the MMA issue work.
 // CTAs 1.. push their fp32 partial sums into landing slots in CTA 0's shared memory with bulk copies
@@ -156,7 +158,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const __grid_constant__ CUtensorMap tmSFA, const __grid_constant__ CUtensorMap tmSFB,
             const __grid_constant__ CUtensorMap tmY, const __grid_constant__ GemmParams p) {
-    using C = GemmCfg<BN, STAGES, PAIR, EPI == kEpiClusterSplit ? kClusterSplitSlots * kClusterSplitSlotBytes : kDefaultOutBytes>;
+    using C = GemmCfg<BN, STAGES, PAIR, cluster_split_slots(EPI) != 0 ? cluster_split_slots(EPI) * kClusterSplitSlotBytes : kDefaultOutBytes>;
     constexpr int ACC = C::ACC;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -174,7 +176,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const uint32_t rank = PAIR ? ptx::cluster_ctarank() : 0u;          // 0 = leader
-    constexpr bool CSPLIT = EPI == kEpiClusterSplit;
+    constexpr bool CSPLIT = EPI == kEpiClusterSplit || EPI == kEpiClusterSplitFew;
     static_assert(!CSPLIT || (BN == 128 && !PAIR && FULLK), "cluster split-K: 128 x 128 tiles, whole K tiles");
     const uint32_t csize = CSPLIT ? static_cast<uint32_t>(p.split_k) : 1u;    // CTAs that share a tile along K
     const uint32_t crank = CSPLIT ? ptx::cluster_ctarank() : 0u;              // which part of K is this CTA's

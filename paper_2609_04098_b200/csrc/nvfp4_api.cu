@@ -257,78 +257,111 @@ nvfp4_status launch_gemm(const GemmMaps& tm, GemmParams& p, int sm_count, cudaSt
 }
 
 // Decode-sized M with fewer 128 x 128 tiles than SMs: clusters of `S` CTAs share a tile along K and
-// meet in the shared memory of the cluster's first CTA (gemm.cuh, kEpiClusterSplit).  Picks the
-// largest S (2..6) for which every tile's cluster is resident at once, every CTA gets at least two
-// K tiles and the partial sums fit the landing slots, and launches; returns NVFP4_ERR_SHAPE without
-// launching when no such S exists -- unless `allow_single` (the caller wants this variant for its
-// in-kernel activation quantization): then S = 1, one CTA per tile, is the fallback.
+// meet in the shared memory of the cluster's first CTA (gemm.cuh, kEpiClusterSplit*).  Two builds of
+// the kernel divide shared memory differently: five stages and two landing slots (a slot holds one
+// CTA's partial sums of one 32-row quarter), or four stages and five slots.
+template <int EPI>
+struct ClusterSplit {
+    static constexpr int BN = 128;
+    static constexpr int STAGES = EPI == kEpiClusterSplitFew ? 5 : 4;
+    static constexpr int SLOTS = cluster_split_slots(EPI);
+    static constexpr int kMaxS = 1 + SLOTS;
+    using C = GemmCfg<BN, STAGES, false, SLOTS * kClusterSplitSlotBytes>;
+
+    static cudaLaunchConfig_t config(cudaLaunchAttribute (&attr)[2], cudaStream_t stream) {
+        cudaLaunchConfig_t cfg;
+        std::memset(&cfg, 0, sizeof(cfg));
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 1;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
+        cfg.blockDim = dim3(kGemmThreads, 1, 1);
+        cfg.dynamicSmemBytes = C::SMEM_BYTES;
+        cfg.stream = stream;
+        cfg.attrs = attr;
+        cfg.numAttrs = 2;
+        return cfg;
+    }
+
+    // The largest S (2..kMaxS) for which every tile's cluster is resident at once, every CTA gets at
+    // least two K tiles and the partial sums fit the slots; 1 if there is none but `allow_single`
+    // (the caller wants this kernel for its in-kernel activation quantization); 0 otherwise, or -1
+    // after a CUDA error.  Sets p.k_per_split for the S it returns.
+    static int plan(GemmParams& p, int sm_count, bool allow_single) {
+        auto kernel = gemm_kernel<BN, STAGES, false, true, EPI>;
+        static std::mutex mu;
+        static std::unordered_map<int, std::array<int, kMaxS + 1>> resident;    // per device and S (0 = unset)
+        int dev = 0;
+        cudaGetDevice(&dev);
+        const int64_t tiles = static_cast<int64_t>(p.m_tiles) * ((p.N + BN - 1) / BN);
+        if (tiles <= 0 || p.m_tiles != 1) return 0;
+        if (tiles * 2 > sm_count && !allow_single) return 0;
+        int S = static_cast<int>(sm_count / tiles);
+        const int live_q = ((p.M < kBM ? p.M : kBM) + 31) / 32;      // 32-row quarters of the tile that hold rows of Y
+        if (S > 1 + SLOTS / live_q) S = 1 + SLOTS / live_q;
+        if (S > p.k_tiles / 2) S = p.k_tiles / 2;
+        {
+            std::lock_guard<std::mutex> lock(mu);
+            auto& r = resident[dev];
+            if (r[0] == 0) {
+                if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
+                    return -1;
+                r[0] = 1;
+            }
+            for (; S >= 2; --S) {
+                if (r[S] == 0) {
+                    cudaLaunchAttribute attr[2];
+                    cudaLaunchConfig_t cfg = config(attr, nullptr);
+                    attr[0].val.clusterDim.x = static_cast<unsigned>(S);
+                    cfg.gridDim = dim3(static_cast<unsigned>(sm_count / S * S), 1, 1);
+                    int n = 0;
+                    if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
+                    r[S] = n > 0 ? n : -1;
+                }
+                if (r[S] >= tiles) break;
+            }
+        }
+        if (S < 1) S = 1;
+        p.k_per_split = (p.k_tiles + S - 1) / S;
+        while (S > 1 && static_cast<int64_t>(S - 1) * p.k_per_split >= p.k_tiles) {          // every CTA has work
+            --S;
+            p.k_per_split = (p.k_tiles + S - 1) / S;
+        }
+        if (S < 2 && !allow_single) return 0;
+        return S;
+    }
+
+    static nvfp4_status launch(const GemmMaps& tm, GemmParams& p, int S, cudaStream_t stream) {
+        auto kernel = gemm_kernel<BN, STAGES, false, true, EPI>;
+        p.n_tiles = (p.N + BN - 1) / BN;
+        p.group_m = p.m_tiles;
+        p.k_per_split = (p.k_tiles + S - 1) / S;
+        p.split_k = S;
+        p.partial = nullptr;
+        p.counters = nullptr;
+        cudaLaunchAttribute attr[2];
+        cudaLaunchConfig_t cfg = config(attr, stream);
+        attr[0].val.clusterDim.x = static_cast<unsigned>(S);
+        cfg.gridDim = dim3(static_cast<unsigned>(static_cast<int64_t>(p.n_tiles) * S), 1, 1);
+        cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, tm.a, tm.b, tm.sfa, tm.sfb, tm.y, p);
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        return e == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+    }
+};
+
+// Launches the cluster-split kernel if the shape takes one: the build with more stages when it
+// splits K as many ways as the other would.  NVFP4_ERR_SHAPE, with nothing launched, if neither applies.
 nvfp4_status launch_gemm_cluster_split(const GemmMaps& tm, GemmParams& p, int sm_count, cudaStream_t stream,
                                        bool allow_single) {
-    constexpr int BN = 128, STAGES = 4, kMaxS = 1 + kClusterSplitSlots;
-    using C = GemmCfg<BN, STAGES, false, kClusterSplitSlots * kClusterSplitSlotBytes>;
-    auto kernel = gemm_kernel<BN, STAGES, false, true, kEpiClusterSplit>;
-    static std::mutex mu;
-    static std::unordered_map<int, std::array<int, kMaxS + 1>> resident;    // per device and S: clusters resident at once (0 = unset)
-    int dev = 0;
-    cudaGetDevice(&dev);
-    p.n_tiles = (p.N + BN - 1) / BN;
-    const int64_t tiles = static_cast<int64_t>(p.m_tiles) * p.n_tiles;
-    if (tiles <= 0 || p.m_tiles != 1) return NVFP4_ERR_SHAPE;
-    if (tiles * 2 > sm_count && !allow_single) return NVFP4_ERR_SHAPE;
-    p.group_m = p.m_tiles;
-    cudaLaunchConfig_t cfg;
-    std::memset(&cfg, 0, sizeof(cfg));
-    cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 1;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
-    cfg.blockDim = dim3(kGemmThreads, 1, 1);
-    cfg.dynamicSmemBytes = C::SMEM_BYTES;
-    cfg.stream = stream;
-    cfg.attrs = attr;
-    cfg.numAttrs = 2;
-    int S = static_cast<int>(sm_count / tiles);
-    const int live_q = ((p.M < kBM ? p.M : kBM) + 31) / 32;      // 32-row quarters of the tile that hold rows of Y
-    if (S > 1 + kClusterSplitSlots / live_q) S = 1 + kClusterSplitSlots / live_q;
-    if (S > p.k_tiles / 2) S = p.k_tiles / 2;
-    {
-        std::lock_guard<std::mutex> lock(mu);
-        auto& r = resident[dev];
-        if (r[0] == 0) {
-            if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
-                return NVFP4_ERR_CUDA;
-            r[0] = 1;
-        }
-        for (; S >= 2; --S) {
-            if (r[S] == 0) {
-                attr[0].val.clusterDim.x = static_cast<unsigned>(S);
-                cfg.gridDim = dim3(static_cast<unsigned>(sm_count / S * S), 1, 1);
-                int n = 0;
-                if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
-                r[S] = n > 0 ? n : -1;
-            }
-            if (r[S] >= tiles) break;
-        }
-    }
-    if (S < 2 && !allow_single) return NVFP4_ERR_SHAPE;
-    if (S < 1) S = 1;
-    p.k_per_split = (p.k_tiles + S - 1) / S;
-    while (S > 1 && static_cast<int64_t>(S - 1) * p.k_per_split >= p.k_tiles) {          // every CTA has work
-        --S;
-        p.k_per_split = (p.k_tiles + S - 1) / S;
-    }
-    if (S < 2 && !allow_single) return NVFP4_ERR_SHAPE;
-    p.split_k = S;
-    p.partial = nullptr;
-    p.counters = nullptr;
-    attr[0].val.clusterDim.x = static_cast<unsigned>(S);
-    cfg.gridDim = dim3(static_cast<unsigned>(tiles * S), 1, 1);
-    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, tm.a, tm.b, tm.sfa, tm.sfb, tm.y, p);
-    g_launches.fetch_add(1, std::memory_order_relaxed);
-    return e == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+    GemmParams few = p, many = p;
+    const int s_few = ClusterSplit<kEpiClusterSplitFew>::plan(few, sm_count, allow_single);
+    const int s_many = ClusterSplit<kEpiClusterSplit>::plan(many, sm_count, allow_single);
+    if (s_few < 0 || s_many < 0) return NVFP4_ERR_CUDA;
+    if (s_few >= 1 && s_few >= s_many) return ClusterSplit<kEpiClusterSplitFew>::launch(tm, p, s_few, stream);
+    if (s_many >= 1) return ClusterSplit<kEpiClusterSplit>::launch(tm, p, s_many, stream);
+    return NVFP4_ERR_SHAPE;
 }
 
 // 128 / 256: one CTA per 128 x BN tile; 2: CTA pair per 256 x 256 tile
