@@ -579,7 +579,7 @@ def run_gpu(args):
                          "traffic": ncu_traffic("quantize_kernel")},
             "calibrate_gbs": round(8192 * HIDDEN * 2 / (cal_ms * 1e-3) / 1e9, 1),
             "rmsnorm_quantize": {"us_per_call": round(rms_ms * 1e3, 2), "value": round(q_bytes / (rms_ms * 1e-3) / 1e9, 1),
-                                 "unit": "GB/s", "note": "RMSNorm fused in front: same HBM bytes, row read twice (second time from cache)"},
+                                 "unit": "GB/s", "note": "RMSNorm fused in front: same HBM bytes, the row stays in registers between the sum of squares and the quantization"},
             "in_step_gbs": None if quant_in_step_gbs is None else round(quant_in_step_gbs, 1)}
         del xq, outs
 

@@ -293,10 +293,12 @@ size_t nvfp4_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int nseg);
  * (paper: Section 9, "Decode overhead" -- activation quantization is the overhead
  * that matters at small batch), codes and scales live in the workspace.
  *   d_x   bf16 [M, K], row stride ldx, 32-byte aligned, ldx % 16 == 0
- * For M = 1 or 2 (single-stream decode) the call is one weight-streaming kernel on the CUDA cores
- * that quantizes the activations itself (same codes) and uses only the status word of the
- * workspace; from M = 3 on it is the quantize kernel followed by the tensor-core GEMM, which starts
- * its prologue while the quantizer still runs.
+ * For M = 1 (and M = 2 where K is not a multiple of 256) the call is one weight-streaming kernel on
+ * the CUDA cores that quantizes the activations itself (same codes); for up to 8 rows with K a
+ * multiple of 256 it is one tensor-core kernel whose CTAs quantize the K tiles of A they multiply
+ * (same codes again); both use only the status word of the workspace.  Above that it is the quantize
+ * kernel followed by the tensor-core GEMM, which starts its prologue while the quantizer still runs.
+ * With NVFP4_W_RESIDENT the GEMM also fetches weights before the work in front of the call is done.
  *   d_workspace  nvfp4_linear_bf16_workspace_bytes(M, N, K, nseg) bytes (status block, split-K
  *                reserve, codes and scales of the activations), 16-byte aligned
  * Every argument is checked before anything is enqueued.

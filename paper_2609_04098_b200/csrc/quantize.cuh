@@ -96,6 +96,32 @@ __device__ __forceinline__ void stg256(void* p, const uint32_t (&v)[8]) {
                  : "memory");
 }
 
+// Two binary32 multiplies (or fused multiply-adds) in one instruction: each half is rounded to nearest
+// even exactly like the scalar instruction, so results are bit-identical and the issue slots halve.
+__device__ __forceinline__ void mul_f32x2(float& a0, float& a1, float b0, float b1) {
+    asm("{\n\t"
+        ".reg .b64 ra, rb;\n\t"
+        "mov.b64 ra, {%0, %1};\n\t"
+        "mov.b64 rb, {%2, %3};\n\t"
+        "mul.rn.f32x2 ra, ra, rb;\n\t"
+        "mov.b64 {%0, %1}, ra;\n\t"
+        "}\n"
+        : "+f"(a0), "+f"(a1)
+        : "f"(b0), "f"(b1));
+}
+// (acc0, acc1) += (a0 * a0, a1 * a1), fused
+__device__ __forceinline__ void fma_sq_f32x2(float& acc0, float& acc1, float a0, float a1) {
+    asm("{\n\t"
+        ".reg .b64 ra, rc;\n\t"
+        "mov.b64 ra, {%2, %3};\n\t"
+        "mov.b64 rc, {%0, %1};\n\t"
+        "fma.rn.f32x2 rc, ra, ra, rc;\n\t"
+        "mov.b64 {%0, %1}, rc;\n\t"
+        "}\n"
+        : "+f"(acc0), "+f"(acc1)
+        : "f"(a0), "f"(a1));
+}
+
 __device__ __forceinline__ uint32_t bf16x2_absmax(uint32_t a, uint32_t b) {
     uint32_t r;
     asm("max.xorsign.abs.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
@@ -121,14 +147,16 @@ __device__ __forceinline__ uint2 quantize_block(const uint32_t (&v)[8], float g,
         float y[8];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            y[2 * i] = __fmul_rn(__uint_as_float(v[i] << 16), q);
-            y[2 * i + 1] = __fmul_rn(__uint_as_float(v[i] & 0xFFFF0000u), q);
+            y[2 * i] = __uint_as_float(v[i] << 16);
+            y[2 * i + 1] = __uint_as_float(v[i] & 0xFFFF0000u);
+            mul_f32x2(y[2 * i], y[2 * i + 1], q, q);
         }
         out.x = f32x8_to_e2m1(y);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            y[2 * i] = __fmul_rn(__uint_as_float(v[4 + i] << 16), q);
-            y[2 * i + 1] = __fmul_rn(__uint_as_float(v[4 + i] & 0xFFFF0000u), q);
+            y[2 * i] = __uint_as_float(v[4 + i] << 16);
+            y[2 * i + 1] = __uint_as_float(v[4 + i] & 0xFFFF0000u);
+            mul_f32x2(y[2 * i], y[2 * i + 1], q, q);
         }
         out.y = f32x8_to_e2m1(y);
     }
@@ -166,8 +194,9 @@ __device__ __forceinline__ void swiglu_block(const uint32_t (&g)[8], const uint3
 __device__ __forceinline__ void rmsnorm_block(const uint32_t (&x)[8], const uint32_t (&w)[8], float rstd, uint32_t (&y)[8]) {
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-        const float lo = __fmul_rn(__fmul_rn(__uint_as_float(x[i] << 16), rstd), __uint_as_float(w[i] << 16));
-        const float hi = __fmul_rn(__fmul_rn(__uint_as_float(x[i] & 0xFFFF0000u), rstd), __uint_as_float(w[i] & 0xFFFF0000u));
+        float lo = __uint_as_float(x[i] << 16), hi = __uint_as_float(x[i] & 0xFFFF0000u);
+        mul_f32x2(lo, hi, rstd, rstd);
+        mul_f32x2(lo, hi, __uint_as_float(w[i] << 16), __uint_as_float(w[i] & 0xFFFF0000u));
         __nv_bfloat162 b2 = __floats2bfloat162_rn(lo, hi);
         y[i] = *reinterpret_cast<uint32_t*>(&b2);
     }
@@ -375,15 +404,15 @@ rmsnorm_quantize_kernel(const uint16_t* __restrict__ x, int32_t M, int32_t rows_
                 for (int e = 0; e < 8; ++e) v[i][e] = 0u;
             }
         }
+        // one pair of partial sums per chunk (independent chains, two squares per instruction), then added up
         float ss = 0.0f;
 #pragma unroll
         for (int i = 0; i < NCH; ++i) {
+            float s0 = 0.0f, s1 = 0.0f;
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                const float lo = __uint_as_float(v[i][e] << 16), hi = __uint_as_float(v[i][e] & 0xFFFF0000u);
-                ss = __fmaf_rn(lo, lo, ss);
-                ss = __fmaf_rn(hi, hi, ss);
-            }
+            for (int e = 0; e < 8; ++e)
+                fma_sq_f32x2(s0, s1, __uint_as_float(v[i][e] << 16), __uint_as_float(v[i][e] & 0xFFFF0000u));
+            ss = __fadd_rn(ss, __fadd_rn(s0, s1));
         }
 #pragma unroll
         for (int off = 16; off >= 1; off >>= 1) ss = __fadd_rn(ss, __shfl_xor_sync(0xffffffffu, ss, off));
