@@ -486,3 +486,54 @@ def test_mlp_chain_with_fused_producer_link_by_link():
     got = oracle.bf16_bits_to_f64(gu.host_bits(y2[rows_t].contiguous()))
     assert np.linalg.norm(got - y2_chain_ref) / np.linalg.norm(y2_chain_ref) <= 3e-3
     assert (hc_ref == hc).mean() > 0.999
+
+
+# ---- kernels that start under their predecessor: a chain of dependent layers, back to back ----------------
+# Every GEMM releases the kernel behind it at once and, with the weights flagged resident, fetches weights
+# while the kernel in front still runs; what it reads from (and writes over) its predecessors is ordered by
+# waits inside the kernels.  A chain in which each layer's input IS the previous layer's output, run back to
+# back on a stream and as a CUDA-graph replay, must give bit for bit what the same chain gives with a device
+# synchronisation after every call -- an ordering mistake shows up as a changed result.
+@pytest.mark.parametrize("M", [4, 64, 300])
+def test_dependent_chain_back_to_back_equals_synchronised(M):
+    K = 2048                                       # square layers: each output feeds the next call
+    depth = 8
+    segs = synth.make_segments((("w", K, 0.02),))
+    ws = nv.alloc_workspace(gu.DEV, M, K, K, 1, fused=True)
+    layers = []
+    for i in range(depth):
+        w_c, w_sf, g_w = nv.nvfp4_quantize_weight(gu.dev_bf16(synth.weights(31, 900 + i, segs, K)), segs)
+        layers.append((w_c, w_sf, g_w))
+    x0 = gu.dev_bf16(synth.activations(31, 1, M, K, n_hot=2, hot_scale=20.0))
+    g_a = gu.dev_f32(np.float32(0.05))            # one static activation scale for every layer
+    bufs = [torch.empty((M, K), dtype=torch.bfloat16, device=gu.DEV) for _ in range(2)]
+    torch.cuda.synchronize()
+
+    def chain(sync):
+        src = x0
+        for i, (w_c, w_sf, g_w) in enumerate(layers):
+            dst = bufs[i & 1]                      # ping-pong: layer i+1 overwrites what layer i read
+            nv.nvfp4_linear_bf16(src, g_a, w_c, w_sf, segs, g_w, ws, out=dst, w_resident=True)
+            if sync:
+                torch.cuda.synchronize()
+            src = dst
+        return src
+
+    want = chain(sync=True).clone()
+    assert nv.device_status(ws) == 0
+    assert bool(torch.isfinite(want.float()).all()) and float(want.float().abs().max()) > 0.0
+    for _ in range(3):
+        got = chain(sync=False)
+        torch.cuda.synchronize()
+        assert torch.equal(got, want)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            out = chain(sync=False)
+        for _ in range(3):
+            graph.replay()
+        side.synchronize()
+    assert torch.equal(out, want)
+    assert nv.device_status(ws) == 0
