@@ -16,7 +16,10 @@
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
+#include <type_traits>
+
 #include "../../include/nvfp4.h"
+#include "ptx.cuh"
 #include "quantize.cuh"
 
 namespace nvfp4 {
@@ -83,15 +86,18 @@ decode_gemv_kernel(const __grid_constant__ DecodeParams p) {
     const int n_slices = (K + 1023) >> 10;
     const int warps_total = gridDim.x * (kDecodeThreads >> 5);
     const bool out_f32 = (p.flags & NVFP4_OUT_F32) != 0u;
-    // a warp's work is a flat list of (row, group of kDecodeSlices slices); the loads of the next
-    // item are issued before the current one is consumed, so the memory latency is paid once
+    // a warp's work is a flat list of (row, group of kDecodeSlices slices); the loads of the next two
+    // items are in flight while the current one is consumed (three register buffers), so a warp with
+    // up to three items -- every warp of a 6144-row layer -- pays the memory latency once
     const int groups = (n_slices + kDecodeSlices - 1) / kDecodeSlices;
     const int first_row = blockIdx.x * (kDecodeThreads >> 5) + warp;
     const int my_rows = first_row < p.N ? (p.N - first_row + warps_total - 1) / warps_total : 0;
     const int items = my_rows * groups;
-    uint4 wv[2][kDecodeSlices];
-    uint32_t sfw[2][kDecodeSlices];
-    auto load_item = [&](int item, int buf) {
+    constexpr int kBufs = 3;
+    uint4 wv[kBufs][kDecodeSlices];
+    uint32_t sfw[kBufs][kDecodeSlices];
+    auto load_item = [&](int item, auto buf_c) {
+        constexpr int buf = decltype(buf_c)::value;
         const int r = item / groups, s0 = (item - r * groups) * kDecodeSlices;
         const int n = first_row + r * warps_total;
         const uint8_t* wrow = p.w_codes + static_cast<int64_t>(n) * (K >> 1);
@@ -108,7 +114,15 @@ decode_gemv_kernel(const __grid_constant__ DecodeParams p) {
             }
         }
     };
-    if (items > 0) load_item(0, 0);
+    // This kernel releases the kernel behind it at once and may itself have been started under its
+    // predecessor: the weights (if the caller flagged them resident) are requested right away, everything
+    // else -- the activations, the global scales, the output -- waits for the predecessor to finish.
+    ptx::pdl_launch_dependents();
+    const bool w_early = (p.flags & NVFP4_W_RESIDENT) != 0u;
+    if (!w_early) ptx::pdl_wait();
+    if (items > 0) load_item(0, std::integral_constant<int, 0>{});
+    if (items > 1) load_item(1, std::integral_constant<int, 1>{});
+    if (w_early) ptx::pdl_wait();
     if (blockIdx.x == 0 && warp == 0) {
         // global scales must be finite and positive; anything else is reported, not repaired
         const float ga = __ldg(p.g_a);
@@ -144,14 +158,11 @@ decode_gemv_kernel(const __grid_constant__ DecodeParams p) {
 
     // ---- 2. stream weight rows
     float acc[MT];
-#pragma unroll 1
-    for (int item = 0; item < items; ++item) {
-        const int buf = item & 1;
+    auto do_item = [&](int item, auto buf_c) {
+        constexpr int buf = decltype(buf_c)::value;
         const int r = item / groups, g0 = item - r * groups, s0 = g0 * kDecodeSlices;
         const int n = first_row + r * warps_total;
-        if (item + 1 < items) {
-            if (buf == 0) load_item(item + 1, 1); else load_item(item + 1, 0);
-        }
+        if (item + 2 < items) load_item(item + 2, std::integral_constant<int, (buf + 2) % kBufs>{});
         if (g0 == 0) {
 #pragma unroll
             for (int m = 0; m < MT; ++m) acc[m] = 0.0f;
@@ -161,8 +172,8 @@ decode_gemv_kernel(const __grid_constant__ DecodeParams p) {
             for (int u = 0; u < kDecodeSlices; ++u) {
                 const int k0 = (s0 + u) * 1024 + lane * 32;
                 if (!(s0 + u < n_slices && k0 < K)) continue;
-                const uint4 wcur = buf == 0 ? wv[0][u] : wv[1][u];
-                const uint32_t scur = buf == 0 ? sfw[0][u] : sfw[1][u];
+                const uint4 wcur = wv[buf][u];
+                const uint32_t scur = sfw[buf][u];
                 // weight scales of the two blocks, weight values as half2
                 uint32_t sh2;
                 asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(sh2) : "h"(static_cast<uint16_t>(scur)));
@@ -211,7 +222,7 @@ decode_gemv_kernel(const __grid_constant__ DecodeParams p) {
                 }
             }
         }
-        if (g0 + 1 < groups) continue;                     // more slices of this row to come
+        if (g0 + 1 < groups) return;                       // more slices of this row to come
         // ---- 3. reduce over lanes, scale, store
 #pragma unroll
         for (int m = 0; m < MT; ++m)
@@ -229,6 +240,12 @@ decode_gemv_kernel(const __grid_constant__ DecodeParams p) {
                 else reinterpret_cast<__nv_bfloat16*>(p.y)[static_cast<int64_t>(m) * p.ldy + n] = __float2bfloat16_rn(v);
             }
         }
+    };
+#pragma unroll 1
+    for (int item = 0; item < items; item += kBufs) {
+        do_item(item, std::integral_constant<int, 0>{});
+        if (item + 1 < items) do_item(item + 1, std::integral_constant<int, 1>{});
+        if (item + 2 < items) do_item(item + 2, std::integral_constant<int, 2>{});
     }
 }
 

@@ -883,9 +883,21 @@ nvfp4_status launch_decode(const DecodeParams& p, int sm_count, cudaStream_t str
     const int64_t rows_per_cta = kDecodeThreads / 32;
     int64_t grid = (p.N + rows_per_cta - 1) / rows_per_cta;
     if (grid > sm_count) grid = sm_count;
-    decode_gemv_kernel<MT><<<static_cast<int>(grid), kDecodeThreads, smem, stream>>>(p);
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof(cfg));
+    cudaLaunchAttribute attr[1];
+    // may start while the kernel in front of it still runs (the kernel itself waits where it has to)
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.gridDim = dim3(static_cast<unsigned>(grid), 1, 1);
+    cfg.blockDim = dim3(kDecodeThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, decode_gemv_kernel<MT>, p);
     g_launches.fetch_add(1, std::memory_order_relaxed);
-    return cudaGetLastError() == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+    return e == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
 
 // workspace of the fused call: [status][split-K reserve][codes][scales]; every part at an offset
