@@ -122,6 +122,10 @@ decode_gemv_kernel(const __grid_constant__ DecodeParams p) {
     if (!w_early) ptx::pdl_wait();
     if (items > 0) load_item(0, std::integral_constant<int, 0>{});
     if (items > 1) load_item(1, std::integral_constant<int, 1>{});
+    // a warp whose whole share fits the three buffers (every warp of a layer with up to 3 x 16 x 148 rows of
+    // up to 5120 elements) takes all its rows at once and reads each activation value once for all of them
+    const bool joint = groups == 1 && items <= kBufs;
+    if (joint && items > 2) load_item(2, std::integral_constant<int, 2>{});
     if (w_early) ptx::pdl_wait();
     if (blockIdx.x == 0 && warp == 0) {
         // global scales must be finite and positive; anything else is reported, not repaired
@@ -157,6 +161,83 @@ decode_gemv_kernel(const __grid_constant__ DecodeParams p) {
     __syncthreads();
 
     // ---- 2. stream weight rows
+    // lane sums of one row -> output values (warp shuffle, global scales, store)
+    auto finish_row = [&](int n, float (&sum)[MT]) {
+#pragma unroll
+        for (int m = 0; m < MT; ++m)
+#pragma unroll
+            for (int off = 16; off >= 1; off >>= 1) sum[m] += __shfl_xor_sync(0xffffffffu, sum[m], off);
+        if (lane == 0) {
+            int sgi = 0;
+            while (sgi + 1 < p.nseg && n >= p.seg_end[sgi]) ++sgi;
+            const float alpha = __fmul_rn(__ldg(p.g_a), __ldg(p.g_seg + sgi));
+#pragma unroll
+            for (int m = 0; m < MT; ++m) {
+                if (m >= p.M) break;
+                const float v = __fmul_rn(sum[m], alpha);
+                if (out_f32) reinterpret_cast<float*>(p.y)[static_cast<int64_t>(m) * p.ldy + n] = v;
+                else reinterpret_cast<__nv_bfloat16*>(p.y)[static_cast<int64_t>(m) * p.ldy + n] = __float2bfloat16_rn(v);
+            }
+        }
+    };
+    if (joint) {
+        // Shared memory is what bounds the row-by-row form: every weight row re-reads the token's values
+        // (10 KB for K = 5120).  Here a 16-byte piece of activations is read once and meets the matching
+        // eight weights of each of the warp's rows, decoded on the spot; same arithmetic per row, same order.
+        float accj[kBufs][MT];
+#pragma unroll
+        for (int b = 0; b < kBufs; ++b)
+#pragma unroll
+            for (int m = 0; m < MT; ++m) accj[b][m] = 0.0f;
+#pragma unroll
+        for (int u = 0; u < kDecodeSlices; ++u) {
+            const int k0 = u * 1024 + lane * 32;
+            if (!(u < n_slices && k0 < K)) continue;
+            const int kb = k0 >> 4;
+#pragma unroll
+            for (int m = 0; m < MT; ++m) {
+                const uint4* ap = reinterpret_cast<const uint4*>(a_val + static_cast<size_t>(m) * KP) +
+                                  (static_cast<size_t>(u) * 4) * 32 + lane;
+                __half2 sum0[kBufs], sum1[kBufs];
+#pragma unroll
+                for (int b = 0; b < kBufs; ++b) { sum0[b] = __float2half2_rn(0.0f); sum1[b] = sum0[b]; }
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const uint4 av = ap[q * 32];
+                    const __half2* a2 = reinterpret_cast<const __half2*>(&av);
+#pragma unroll
+                    for (int b = 0; b < kBufs; ++b) {
+                        if (b >= items) break;                                   // warp-uniform
+                        const uint32_t word = q == 0 ? wv[b][u].x : (q == 1 ? wv[b][u].y : (q == 2 ? wv[b][u].z : wv[b][u].w));
+                        __half2 t[4];
+                        e2m1x8_to_half2x4(word, t);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            if (q < 2) sum0[b] = __hfma2(a2[e], t[e], sum0[b]);
+                            else       sum1[b] = __hfma2(a2[e], t[e], sum1[b]);
+                        }
+                    }
+                }
+                const float2 sa = *reinterpret_cast<const float2*>(a_scale + m * KB + kb);     // kb is even
+#pragma unroll
+                for (int b = 0; b < kBufs; ++b) {
+                    if (b >= items) break;
+                    uint32_t sh2;
+                    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(sh2) : "h"(static_cast<uint16_t>(sfw[b][u])));
+                    const float2 sw = __half22float2(*reinterpret_cast<__half2*>(&sh2));
+                    const float2 b0 = __half22float2(sum0[b]), b1 = __half22float2(sum1[b]);
+                    accj[b][m] = __fmaf_rn(__fadd_rn(b0.x, b0.y), __fmul_rn(sa.x, sw.x), accj[b][m]);
+                    accj[b][m] = __fmaf_rn(__fadd_rn(b1.x, b1.y), __fmul_rn(sa.y, sw.y), accj[b][m]);
+                }
+            }
+        }
+#pragma unroll
+        for (int b = 0; b < kBufs; ++b) {
+            if (b >= items) break;
+            finish_row(first_row + b * warps_total, accj[b]);
+        }
+        return;
+    }
     float acc[MT];
     auto do_item = [&](int item, auto buf_c) {
         constexpr int buf = decltype(buf_c)::value;
@@ -224,22 +305,7 @@ decode_gemv_kernel(const __grid_constant__ DecodeParams p) {
         }
         if (g0 + 1 < groups) return;                       // more slices of this row to come
         // ---- 3. reduce over lanes, scale, store
-#pragma unroll
-        for (int m = 0; m < MT; ++m)
-#pragma unroll
-            for (int off = 16; off >= 1; off >>= 1) acc[m] += __shfl_xor_sync(0xffffffffu, acc[m], off);
-        if (lane == 0) {
-            int sgi = 0;
-            while (sgi + 1 < p.nseg && n >= p.seg_end[sgi]) ++sgi;
-            const float alpha = __fmul_rn(__ldg(p.g_a), __ldg(p.g_seg + sgi));
-#pragma unroll
-            for (int m = 0; m < MT; ++m) {
-                if (m >= p.M) break;
-                const float v = __fmul_rn(acc[m], alpha);
-                if (out_f32) reinterpret_cast<float*>(p.y)[static_cast<int64_t>(m) * p.ldy + n] = v;
-                else reinterpret_cast<__nv_bfloat16*>(p.y)[static_cast<int64_t>(m) * p.ldy + n] = __float2bfloat16_rn(v);
-            }
-        }
+        finish_row(n, acc);
     };
 #pragma unroll 1
     for (int item = 0; item < items; item += kBufs) {
