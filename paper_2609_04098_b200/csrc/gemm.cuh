@@ -653,6 +653,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     }
                     continue;
                 }
+                // CTA 0.  While the other CTAs' copies are on their way (about 1 000 cycles for 16 KB) the
+                // per-column global scales go into a small table in the stage area (idle by now), from where
+                // they come back as broadcast reads (a shuffle per column costs more than the whole sum).
+                const uint32_t scale_tab = ptx::smem_u32(smem) + static_cast<uint32_t>(quarter) * (BN * 4);
+                if (quarter_live) {
+#pragma unroll
+                    for (int i = 0; i < BN / 32; ++i) ptx::st_shared_f32(scale_tab + static_cast<uint32_t>((i * 32 + lane) * 4), areg[i]);
+                    __syncwarp();                                  // the table is complete before any lane reads it
+                }
                 if (lane == 0) ok = ptx::mbar_wait_bounded(cs_ready, 0u, abort_flag, p.wait_limit_ns, 0u);
                 ok = __shfl_sync(0xffffffffu, static_cast<int>(ok), 0) != 0;
                 if (!ok) break;
@@ -681,8 +690,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                         }
                     }
 #pragma unroll
-                    for (int j = 0; j < 64; ++j)
-                        v[j] = __fmul_rn(v[j], __shfl_sync(0xffffffffu, areg[pc * 2 + (j >> 5)], j & 31));
+                    for (int j = 0; j < 16; ++j) {
+                        const uint4 sc = ptx::ld_shared_v4(scale_tab + static_cast<uint32_t>((pc * kOutPieceCols + 4 * j) * 4));
+                        v[4 * j] = __fmul_rn(v[4 * j], __uint_as_float(sc.x));
+                        v[4 * j + 1] = __fmul_rn(v[4 * j + 1], __uint_as_float(sc.y));
+                        v[4 * j + 2] = __fmul_rn(v[4 * j + 2], __uint_as_float(sc.z));
+                        v[4 * j + 3] = __fmul_rn(v[4 * j + 3], __uint_as_float(sc.w));
+                    }
                     if (use_tma) {
                         // this piece's part of the first landing slot of this quarter is in registers by now:
                         // it serves as the staging buffer of the TMA store (rows past M are clipped there)
@@ -835,7 +849,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             if (C::OVERLAP && acc == 0u) drain(std::integral_constant<int, NP - 1>{});
             else                         drain(std::integral_constant<int, 0>{});
         }
-        if (use_tma && lane == 0) ptx::bulk_wait_group<0>();   // all output stores complete before exit
+        // every output store has read its shared-memory source before the CTA goes away (the writes
+        // themselves are complete, like any other global write, when the kernel is)
+        if (use_tma && lane == 0) ptx::bulk_wait_group_read<0>();
     }
 
     // ---------------------------------------------------------------- teardown
