@@ -141,7 +141,7 @@ __device__ __forceinline__ uint2 quantize_block(const uint32_t (&v)[8], float g,
     const uint32_t s8 = f32_to_e4m3(__fmul_rn(bmax, c1));
     s8_out = s8;
     const float d = __fmul_rn(e4m3_to_f32(s8), g);
-    const float q = __fdiv_rn(1.0f, d);                       // s8 == 0 gives inf; that block is zeroed below
+    const float q = __frcp_rn(d);                             // the correctly rounded 1 / d (s8 == 0 gives inf; that block is zeroed below)
     uint2 out;
     {
         float y[8];
