@@ -324,7 +324,7 @@ def test_long_prefill_32k_tokens_sampled():
 # 8 tokens (K a multiple of 256): one tensor-core kernel that quantizes the activations itself; otherwise quantize
 # kernel + GEMM
 @pytest.mark.parametrize("M", [1, 2, 3, 4, 8, 9, 16, 17])
-@pytest.mark.parametrize("N,K", [(6144, 5120), (1000, 1088), (5120, 17408), (50, 64), (34816, 512)])
+@pytest.mark.parametrize("N,K", [(6144, 5120), (1000, 1088), (5120, 17408), (50, 64), (34816, 512), (300, 256), (129, 768)])
 @pytest.mark.parametrize("out_f32", [False, True])
 def test_decode_batches(M, N, K, out_f32):
     n1 = max(1, N // 3)
