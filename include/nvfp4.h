@@ -392,7 +392,8 @@ nvfp4_status nvfp4_gdn_lockstep(const float* d_q, const float* d_k, const float*
 /*
  * Measurement aid: the SM clock the last tensor-core GEMM launched on this workspace really ran at
  * (its first CTA's cycle counter over the wall clock, both read inside the kernel and left in the
- * status block), and that CTA's lifetime in microseconds.  Under a power cap the clock drops within
+ * status block), and that CTA's lifetime in microseconds -- from its start, which may lie under the
+ * tail of the kernel in front of it, to its end.  Under a power cap the clock drops within
  * microseconds, long before a management-library sample shows it.  Synchronises `stream`.
  */
 nvfp4_status nvfp4_last_gemm_clock(const void* d_workspace, double* sm_mhz, double* kernel_us, void* stream);
