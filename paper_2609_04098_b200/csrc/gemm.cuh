@@ -94,7 +94,8 @@ constexpr int kOutPieceBytes = 32 * kOutPieceCols * 2;
 constexpr int kClusterSplitSlotBytes = 32 * 128 * 4;      // fp32 partial sums of one 32-row quarter of a 128-wide tile
 // landing slots in the cluster's first CTA: five beside four stages, or two beside five stages
 __host__ __device__ constexpr int cluster_split_slots(int epi) { return epi == 2 ? 5 : (epi == 3 ? 2 : 0); }
-constexpr int kDefaultOutBytes = 4 * 2 * kOutPieceBytes;  // per epilogue warp: two pieces
+constexpr int kScaleTabBytes = 4 * kOutPieceCols * 4;     // per epilogue warp: the global scales of one piece's columns
+constexpr int kDefaultOutBytes = 4 * 2 * kOutPieceBytes + kScaleTabBytes;  // per epilogue warp: two pieces, and the scale table
 
 template <int BN, int STAGES, bool PAIR, int OUT_BYTES_ = kDefaultOutBytes>
 struct GemmCfg {
@@ -782,6 +783,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             }
             // piece order: with overlapping accumulators the shared columns go first (the last piece
             // of the lower accumulator, the first piece of the upper one)
+            const uint32_t scale_tab = ptx::smem_u32(out_s) + 4 * 2 * kOutPieceBytes + static_cast<uint32_t>(quarter) * (kOutPieceCols * 4);
             auto drain = [&](auto first_c) {
             constexpr int first_piece = decltype(first_c)::value;
             uint32_t ra[64], rb[64];
@@ -805,10 +807,22 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 }
                 const int32_t col0 = n0 + pc * kOutPieceCols;
                 if (col0 >= p.N || row0 >= p.M) continue;        // warp-uniform
+                // the 64 column scales of this piece go through a 256-byte table in shared memory and come
+                // back as broadcast reads: 2 stores + 16 loads per lane instead of 64 shuffles (this warp
+                // shares its scheduler with a producer or with the warp that issues the MMAs)
                 float v[64];
+                __syncwarp();
+                ptx::st_shared_f32(scale_tab + static_cast<uint32_t>(lane * 4), areg[pc * 2]);
+                ptx::st_shared_f32(scale_tab + static_cast<uint32_t>(128 + lane * 4), areg[pc * 2 + 1]);
+                __syncwarp();
 #pragma unroll
-                for (int j = 0; j < 64; ++j)
-                    v[j] = __fmul_rn(__uint_as_float(cur[j]), __shfl_sync(0xffffffffu, areg[pc * 2 + (j >> 5)], j & 31));
+                for (int j = 0; j < 16; ++j) {
+                    const uint4 sc = ptx::ld_shared_v4(scale_tab + static_cast<uint32_t>(j * 16));
+                    v[4 * j] = __fmul_rn(__uint_as_float(cur[4 * j]), __uint_as_float(sc.x));
+                    v[4 * j + 1] = __fmul_rn(__uint_as_float(cur[4 * j + 1]), __uint_as_float(sc.y));
+                    v[4 * j + 2] = __fmul_rn(__uint_as_float(cur[4 * j + 2]), __uint_as_float(sc.z));
+                    v[4 * j + 3] = __fmul_rn(__uint_as_float(cur[4 * j + 3]), __uint_as_float(sc.w));
+                }
                 if (use_tma) {
                     uint8_t* buf = out_w + (pieces_stored & 1u) * kOutPieceBytes;
                     if (pieces_stored >= 2u) {
