@@ -818,10 +818,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
                     const uint4 sc = ptx::ld_shared_v4(scale_tab + static_cast<uint32_t>(j * 16));
-                    v[4 * j] = __fmul_rn(__uint_as_float(cur[4 * j]), __uint_as_float(sc.x));
-                    v[4 * j + 1] = __fmul_rn(__uint_as_float(cur[4 * j + 1]), __uint_as_float(sc.y));
-                    v[4 * j + 2] = __fmul_rn(__uint_as_float(cur[4 * j + 2]), __uint_as_float(sc.z));
-                    v[4 * j + 3] = __fmul_rn(__uint_as_float(cur[4 * j + 3]), __uint_as_float(sc.w));
+                    v[4 * j] = __uint_as_float(cur[4 * j]);
+                    v[4 * j + 1] = __uint_as_float(cur[4 * j + 1]);
+                    v[4 * j + 2] = __uint_as_float(cur[4 * j + 2]);
+                    v[4 * j + 3] = __uint_as_float(cur[4 * j + 3]);
+                    mul_f32x2(v[4 * j], v[4 * j + 1], __uint_as_float(sc.x), __uint_as_float(sc.y));       // two products per instruction
+                    mul_f32x2(v[4 * j + 2], v[4 * j + 3], __uint_as_float(sc.z), __uint_as_float(sc.w));
                 }
                 if (use_tma) {
                     uint8_t* buf = out_w + (pieces_stored & 1u) * kOutPieceBytes;
