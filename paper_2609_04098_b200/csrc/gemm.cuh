@@ -559,12 +559,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                         uint32_t hw[8];
 #pragma unroll
                         for (int i = 0; i < 8; ++i) {
-                            // gate / up rounded to bf16 exactly as the plain epilogue would store them
-                            const float g0 = __bfloat162float(__float2bfloat16_rn(__fmul_rn(__uint_as_float(cur[b * 32 + 2 * i]), a_gate)));
-                            const float g1 = __bfloat162float(__float2bfloat16_rn(__fmul_rn(__uint_as_float(cur[b * 32 + 2 * i + 1]), a_gate)));
-                            const float u0 = __bfloat162float(__float2bfloat16_rn(__fmul_rn(__uint_as_float(cur[b * 32 + 16 + 2 * i]), a_up)));
-                            const float u1 = __bfloat162float(__float2bfloat16_rn(__fmul_rn(__uint_as_float(cur[b * 32 + 16 + 2 * i + 1]), a_up)));
-                            hw[i] = pack_bf16x2(silu_mul(g0, u0), silu_mul(g1, u1));
+                            // gate / up rounded to bf16 exactly as the plain epilogue would store them (two values per
+                            // multiply and per rounding instruction; the rounded pair is unpacked again by shift and mask)
+                            float g0 = __uint_as_float(cur[b * 32 + 2 * i]), g1 = __uint_as_float(cur[b * 32 + 2 * i + 1]);
+                            float u0 = __uint_as_float(cur[b * 32 + 16 + 2 * i]), u1 = __uint_as_float(cur[b * 32 + 16 + 2 * i + 1]);
+                            mul_f32x2(g0, g1, a_gate, a_gate);
+                            mul_f32x2(u0, u1, a_up, a_up);
+                            const uint32_t gb = pack_bf16x2(g0, g1), ub = pack_bf16x2(u0, u1);
+                            float h0, h1;
+                            silu_mul2(__uint_as_float(gb << 16), __uint_as_float(gb & 0xFFFF0000u), __uint_as_float(ub << 16),
+                                      __uint_as_float(ub & 0xFFFF0000u), h0, h1);
+                            hw[i] = pack_bf16x2(h0, h1);
                         }
                         words[b] = quantize_block(hw, g_h, c1_h, s8[b]);
                         if (p.dbg_h != nullptr && row < p.M)

@@ -179,12 +179,40 @@ __device__ __forceinline__ float silu_mul(float g, float u) {
     return __fmul_rn(__fmul_rn(g, r), u);
 }
 
+// The same for two elements at once: the three multiplies and the add are issued as two-wide binary32
+// instructions (each half rounded exactly like the scalar form: the results are bit-identical).
+__device__ __forceinline__ void add_f32x2(float& a0, float& a1, float b0, float b1) {
+    asm("{\n\t"
+        ".reg .b64 ra, rb;\n\t"
+        "mov.b64 ra, {%0, %1};\n\t"
+        "mov.b64 rb, {%2, %3};\n\t"
+        "add.rn.f32x2 ra, ra, rb;\n\t"
+        "mov.b64 {%0, %1}, ra;\n\t"
+        "}\n"
+        : "+f"(a0), "+f"(a1)
+        : "f"(b0), "f"(b1));
+}
+__device__ __forceinline__ void silu_mul2(float g0, float g1, float u0, float u1, float& h0, float& h1) {
+    float t0 = g0, t1 = g1, e0, e1, r0, r1;
+    mul_f32x2(t0, t1, -1.44269504088896341f, -1.44269504088896341f);
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"(t0));
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"(t1));
+    add_f32x2(e0, e1, 1.0f, 1.0f);
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r0) : "f"(e0));
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r1) : "f"(e1));
+    h0 = g0;
+    h1 = g1;
+    mul_f32x2(h0, h1, r0, r1);
+    mul_f32x2(h0, h1, u0, u1);
+}
+
 // 16 gate values and 16 up values (packed bf16) -> 16 values of bf16(silu(gate) * up), packed
 __device__ __forceinline__ void swiglu_block(const uint32_t (&g)[8], const uint32_t (&u)[8], uint32_t (&h)[8]) {
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-        const float lo = silu_mul(__uint_as_float(g[i] << 16), __uint_as_float(u[i] << 16));
-        const float hi = silu_mul(__uint_as_float(g[i] & 0xFFFF0000u), __uint_as_float(u[i] & 0xFFFF0000u));
+        float lo, hi;
+        silu_mul2(__uint_as_float(g[i] << 16), __uint_as_float(g[i] & 0xFFFF0000u), __uint_as_float(u[i] << 16),
+                  __uint_as_float(u[i] & 0xFFFF0000u), lo, hi);
         __nv_bfloat162 b2 = __floats2bfloat162_rn(lo, hi);
         h[i] = *reinterpret_cast<uint32_t*>(&b2);
     }
