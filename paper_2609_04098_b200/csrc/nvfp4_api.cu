@@ -102,18 +102,48 @@ struct MapKeyHash {
     }
 };
 
+// Encoded tensor maps by (pointer, shape).  A map costs about a microsecond of host time to encode; a
+// loop over the same buffers (a model's weights, a server's ring of activation buffers) never encodes
+// twice.  A caller that hands in fresh pointers for ever fills the table: when it is full the older
+// half of the entries goes (by insertion stamp), not the entries that are in use.
+class MapCache {
+public:
+    bool find(const MapKey& key, CUtensorMap* out) {
+        std::lock_guard<std::mutex> lock(mu_);
+        auto it = map_.find(key);
+        if (it == map_.end()) return false;
+        *out = it->second.map;
+        return true;
+    }
+    void insert(const MapKey& key, const CUtensorMap& m) {
+        std::lock_guard<std::mutex> lock(mu_);
+        if (map_.size() >= kCapacity) {
+            const uint64_t cut = stamp_ - kCapacity / 2;
+            for (auto it = map_.begin(); it != map_.end();) {
+                if (it->second.stamp < cut) it = map_.erase(it); else ++it;
+            }
+        }
+        map_[key] = Entry{m, stamp_++};
+    }
+
+private:
+    static constexpr size_t kCapacity = 4096;
+    struct Entry {
+        CUtensorMap map;
+        uint64_t stamp;
+    };
+    std::mutex mu_;
+    std::unordered_map<MapKey, Entry, MapKeyHash> map_;
+    uint64_t stamp_ = kCapacity;
+};
+
 // codes [rows, K/2] bytes, tiles of box_rows x 128 bytes, 128-byte swizzle, zero fill outside
 nvfp4_status codes_tensor_map(const uint8_t* d_codes, int64_t rows, int64_t K, int box_rows, CUtensorMap* out) {
-    static std::mutex mu;
-    static std::unordered_map<MapKey, CUtensorMap, MapKeyHash> cache;
+    static MapCache cache;
     int dev = 0;
     cudaGetDevice(&dev);
     MapKey key{d_codes, rows, K / 2, box_rows, dev};
-    {
-        std::lock_guard<std::mutex> lock(mu);
-        auto it = cache.find(key);
-        if (it != cache.end()) { *out = it->second; return NVFP4_OK; }
-    }
+    if (cache.find(key, out)) return NVFP4_OK;
     EncodeTiledFn enc = encode_fn();
     if (enc == nullptr) return NVFP4_ERR_CUDA;
     const cuuint64_t dims[2] = {static_cast<cuuint64_t>(K / 2), static_cast<cuuint64_t>(rows)};
@@ -124,26 +154,19 @@ nvfp4_status codes_tensor_map(const uint8_t* d_codes, int64_t rows, int64_t K, i
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return NVFP4_ERR_CUDA;
-    std::lock_guard<std::mutex> lock(mu);
-    if (cache.size() > 4096) cache.clear();
-    cache[key] = *out;
+    cache.insert(key, *out);
     return NVFP4_OK;
 }
 
 // scale bytes in the tensor-core layout seen as [band][k-atom][128 x u32]; a box takes four
 // k-atoms of `box_bands` bands; bands and k-atoms past the tensor read as zero
 nvfp4_status scales_tensor_map(const uint8_t* d_sf, int64_t rows, int64_t K, int box_bands, CUtensorMap* out) {
-    static std::mutex mu;
-    static std::unordered_map<MapKey, CUtensorMap, MapKeyHash> cache;
+    static MapCache cache;
     int dev = 0;
     cudaGetDevice(&dev);
     const int64_t bands = (rows + 127) / 128, katoms = K / 64;
     MapKey key{d_sf, bands, katoms, box_bands, dev};
-    {
-        std::lock_guard<std::mutex> lock(mu);
-        auto it = cache.find(key);
-        if (it != cache.end()) { *out = it->second; return NVFP4_OK; }
-    }
+    if (cache.find(key, out)) return NVFP4_OK;
     EncodeTiledFn enc = encode_fn();
     if (enc == nullptr) return NVFP4_ERR_CUDA;
     const cuuint64_t dims[3] = {128, static_cast<cuuint64_t>(katoms), static_cast<cuuint64_t>(bands)};
@@ -154,24 +177,17 @@ nvfp4_status scales_tensor_map(const uint8_t* d_sf, int64_t rows, int64_t K, int
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return NVFP4_ERR_CUDA;
-    std::lock_guard<std::mutex> lock(mu);
-    if (cache.size() > 4096) cache.clear();
-    cache[key] = *out;
+    cache.insert(key, *out);
     return NVFP4_OK;
 }
 
 // bf16 output [M, N] with row stride ldy, 32 x 64 boxes, 128-byte swizzle (TMA stores clip at M and N)
 nvfp4_status output_tensor_map(void* d_y, int64_t M, int64_t N, int64_t ldy, CUtensorMap* out) {
-    static std::mutex mu;
-    static std::unordered_map<MapKey, CUtensorMap, MapKeyHash> cache;
+    static MapCache cache;
     int dev = 0;
     cudaGetDevice(&dev);
     MapKey key{d_y, M, N * 4096 + (ldy % 4096), static_cast<int>(ldy / 4096), dev};
-    {
-        std::lock_guard<std::mutex> lock(mu);
-        auto it = cache.find(key);
-        if (it != cache.end()) { *out = it->second; return NVFP4_OK; }
-    }
+    if (cache.find(key, out)) return NVFP4_OK;
     EncodeTiledFn enc = encode_fn();
     if (enc == nullptr) return NVFP4_ERR_CUDA;
     const cuuint64_t dims[2] = {static_cast<cuuint64_t>(N), static_cast<cuuint64_t>(M)};
@@ -182,9 +198,7 @@ nvfp4_status output_tensor_map(void* d_y, int64_t M, int64_t N, int64_t ldy, CUt
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return NVFP4_ERR_CUDA;
-    std::lock_guard<std::mutex> lock(mu);
-    if (cache.size() > 4096) cache.clear();
-    cache[key] = *out;
+    cache.insert(key, *out);
     return NVFP4_OK;
 }
 

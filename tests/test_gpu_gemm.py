@@ -537,3 +537,24 @@ def test_dependent_chain_back_to_back_equals_synchronised(M):
         side.synchronize()
     assert torch.equal(out, want)
     assert nv.device_status(ws) == 0
+
+
+# ---- more distinct output buffers than the table of encoded tensor maps holds ------------------------------
+def test_many_distinct_output_pointers():
+    M, N, K = 130, 64, 64                                   # the TMA-store path (bf16, aligned rows)
+    segs, x, w, ac, asf, ga, wc, wsf, gs = _oracle_operands(41, M, K, (("p", N, 0.02),))
+    y_ref = oracle.gemm(ac, asf, ga, wc, wsf, oracle.col_scales(N, segs, gs))
+    bound = gu.gemm_bounds(ac, asf, ga, wc, wsf, oracle.col_scales(N, segs, gs))
+    a_c, a_sf, g_a = gu.dev_u8(ac), gu.dev_u8(oracle.sf_to_mma(asf, K)), gu.dev_f32(ga)
+    w_c, w_sf, g_w = gu.dev_u8(wc), gu.dev_u8(oracle.sf_to_mma(wsf, K)), gu.dev_f32(gs)
+    ws = _ws()
+    n_bufs = 4500
+    pool = torch.zeros((n_bufs, M, N), dtype=torch.bfloat16, device=gu.DEV)
+    for i in range(n_bufs):
+        nv.nvfp4_linear(a_c, a_sf, g_a, w_c, w_sf, segs, g_w, ws, out=pool[i])
+    nv.nvfp4_linear(a_c, a_sf, g_a, w_c, w_sf, segs, g_w, ws, out=pool[0])     # an entry that was evicted long ago
+    torch.cuda.synchronize()
+    assert nv.device_status(ws) == 0
+    for i in (0, 1, 2047, 2048, 4095, 4096, n_bufs - 1):
+        gu.check_gemm(pool[i], y_ref, bound, "buffer %d" % i)
+    assert torch.equal(pool[0], pool[n_bufs - 1]) and torch.equal(pool[17], pool[4321])
